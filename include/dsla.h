@@ -1,0 +1,171 @@
+/*
+ * libdsla -- dual-state linear attention (DSLA) layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer replaces softmax self-attention at inference time.  Per (sequence, head) it keeps two
+ * recurrent states, "history" (i = 1, slow decay) and "recency" (i = 2, fast decay):
+ *
+ *     S^i_t = g^i_t * S^i_{t-1} + k_t^T v_t                      (Sec. 4.1, dual-state update)
+ *     o_t   = scale * q_t ( gamma S^1_t + (1 - gamma) S^2_t )    (Sec. 4.1, blended readout)
+ *
+ * g^i_t in [0,1] is an already-activated scalar gate per (token, head, state); gamma is a blend
+ * weight per head (a per-layer gamma is the same value in every entry).  The feature map is the
+ * identity and there is no normaliser (none is defined in Sec. 4.1).
+ *
+ * Conventions for every entry point
+ *   - plain C ABI; every pointer is a DEVICE pointer unless its comment says "host";
+ *   - the caller owns all tensors; prefill and decode allocate nothing;
+ *   - work is enqueued on the CUDA stream passed as `cuda_stream` (a cudaStream_t; NULL = default
+ *     stream) and the call returns without waiting for it;
+ *   - argument errors are detected on the host before anything is launched and reported through
+ *     the return value; nothing is thrown, nothing aborts, there is no CPU fallback;
+ *   - supported head sizes: d_k == d_v in {64, 128}; everything else is DSLA_ERR_UNSUPPORTED.
+ */
+#ifndef DSLA_H_
+#define DSLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DSLA_OK = 0,
+    DSLA_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, misaligned pointer, slot out of range ... */
+    DSLA_ERR_UNSUPPORTED = 2, /* head size / chunk / dtype combination that no kernel covers */
+    DSLA_ERR_CUDA = 3,        /* a CUDA runtime call failed (no device, launch error, ...) */
+    DSLA_ERR_OOM = 4,         /* device allocation failed (dsla_state_alloc only) */
+    DSLA_ERR_TIMEOUT = 5      /* a bounded on-device wait ran out; see dsla_state_last_error */
+} dsla_status;
+
+typedef enum { DSLA_F32 = 0, DSLA_BF16 = 1 } dsla_dtype;
+
+/* Which prefill kernel runs.  AUTO picks TENSOR for bf16 with d = 128 and SIMT otherwise. */
+typedef enum { DSLA_IMPL_AUTO = 0, DSLA_IMPL_SIMT = 1, DSLA_IMPL_TENSOR = 2 } dsla_impl;
+
+/* ------------------------------------------------------------------------------------------
+ * Dual-state store.  One "slot" holds the two states of every head of one sequence of one layer:
+ * fp32 [num_slots][2][H][d_k][d_v], d_v contiguous; index 0 of the second axis is the history
+ * state S^1, index 1 the recency state S^2 (the two states of Sec. 4.1).  Its size does not depend
+ * on the context length (Sec. 5.3: decoding updates only two states).
+ * ------------------------------------------------------------------------------------------ */
+typedef struct dsla_state dsla_state;
+
+/* Bytes needed for the store above (0 on invalid sizes). */
+size_t dsla_state_bytes(int num_slots, int H, int d_k, int d_v);
+
+/* Creates a store on the current device.
+ *   ext_buf == NULL : the library cudaMalloc's dsla_state_bytes() once (DSLA_ERR_OOM on failure);
+ *   ext_buf != NULL : the store borrows caller memory (256-byte aligned, ext_bytes >= the size
+ *                     above, else DSLA_ERR_INVALID_ARG); the caller keeps ownership.
+ * The contents are NOT initialised; call dsla_state_zero or run a prefill with
+ * use_initial_state = 0.  A 4-byte device status word is allocated alongside. */
+dsla_status dsla_state_alloc(dsla_state** out, int num_slots, int H, int d_k, int d_v,
+                             void* ext_buf, size_t ext_bytes);
+
+/* Frees the handle and only the memory the library allocated.  NULL is accepted. */
+dsla_status dsla_state_free(dsla_state* st);
+
+/* Device pointer to the fp32 store (for copy-out, checkpointing, parity checks). */
+void* dsla_state_data(dsla_state* st);
+
+/* Zeroes n slots listed in slots_dev (device int32[n]; entries < 0 are ignored), or the whole
+ * store when slots_dev == NULL (n is then ignored). */
+dsla_status dsla_state_zero(dsla_state* st, const int32_t* slots_dev, int n, void* cuda_stream);
+
+/* Reads back (synchronising the whole device) and clears the status word that kernels set when a
+ * bounded wait gives up: DSLA_OK or DSLA_ERR_TIMEOUT. */
+dsla_status dsla_state_last_error(dsla_state* st);
+
+/* ------------------------------------------------------------------------------------------
+ * Prefill: the chunkwise-parallel form of the recurrence.  Inside a chunk of C tokens the output
+ * is the masked quadratic form of the unrolled scores (Sec. 4.1: sigma^i_t = (q_T . k_t) times the
+ * product of the gates t+1..T, blended by gamma); between chunks the two states are carried as
+ *     S^i <- (prod of the chunk's gates) S^i + sum_s (prod of gates s+1..end) k_s^T v_s .
+ * The result equals the token-by-token recurrence up to floating-point summation order and does
+ * not depend on `chunk`.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    const void* q;              /* [T_total, H, d_k]  dtype, row-major, 16-byte aligned           */
+    const void* k;              /* [T_total, H, d_k]                                              */
+    const void* v;              /* [T_total, H, d_v]                                              */
+    void* o;                    /* [T_total, H, d_v]  dtype (output)                              */
+    const float* g_hist;        /* [T_total, H] fp32 in [0,1]: gate of the history state          */
+    const float* g_rec;         /* [T_total, H] fp32 in [0,1]: gate of the recency state          */
+    const float* gamma;         /* [H] fp32: weight of the history branch; recency gets 1 - gamma */
+    const int32_t* cu_seqlens;  /* [N + 1] int32, cu[0] = 0, cu[N] = T_total (packed sequences);
+                                   NULL means N sequences of exactly T tokens each               */
+    const int32_t* slots;       /* [N] int32 slot of each sequence; NULL means slot n = n.  Entries
+                                   must be distinct and in [0, num_slots) (not checked on host)  */
+    int N;                      /* number of sequences                                           */
+    int T;                      /* tokens per sequence when cu_seqlens == NULL, else ignored      */
+    int T_total;                /* rows of q/k/v/o                                               */
+    int max_seqlen;             /* upper bound on any sequence length (sizes the grid)           */
+    int H, d_k, d_v;
+    int chunk;                  /* C: 16, 32 or 64 for the SIMT kernel; 64 (or 0 = default) for
+                                   the tensor-core kernel, which tiles two chunks per MMA tile   */
+    dsla_dtype dtype;           /* dtype of q, k, v, o; the states are always fp32               */
+    float scale;                /* multiplies o (1.0f for the plain definition)                  */
+    int use_initial_state;      /* 0: start every sequence from zero states; 1: continue from the
+                                   contents of its slot (chunked prefill / resume)               */
+    dsla_impl impl;
+    void* workspace;            /* scratch of dsla_prefill_workspace_bytes(); may be NULL if 0    */
+    size_t workspace_bytes;
+} dsla_prefill_args;
+
+/* Scratch the chosen kernel needs for these sizes (0 for the SIMT kernel).  Pointers in `a` are
+ * not dereferenced. */
+size_t dsla_prefill_workspace_bytes(const dsla_prefill_args* a);
+
+/* Writes o for every token and the final states of every sequence into its slot.  A sequence of
+ * length 0 writes no output; its slot is zeroed when use_initial_state == 0 and left as is
+ * otherwise.  `a` is a host pointer and is read before the call returns. */
+dsla_status dsla_prefill(const dsla_prefill_args* a, dsla_state* st, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Decode: one step of the recurrence per batch row, fused with the readout and the blend
+ * (Sec. 4.1 equations applied to one new token; Sec. 5.3: constant cost per token).  Each state
+ * element is read once and written once, in place.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    const void* q;          /* [B, H, d_k] dtype                                                  */
+    const void* k;          /* [B, H, d_k]                                                        */
+    const void* v;          /* [B, H, d_v]                                                        */
+    void* o;                /* [B, H, d_v] dtype (output); rows with slot < 0 are written as 0    */
+    const float* g_hist;    /* [B, H] fp32                                                        */
+    const float* g_rec;     /* [B, H] fp32                                                        */
+    const float* gamma;     /* [H] fp32                                                           */
+    const int32_t* slots;   /* [B] int32 slot per row; < 0 skips the row (padding in a continuous
+                               batch); NULL means slot b = b.  Live entries must be distinct     */
+    int B, H, d_k, d_v;
+    dsla_dtype dtype;
+    float scale;
+} dsla_decode_args;
+
+dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * Host-buffer variants (end-to-end path): q, k, v, o, g_hist, g_rec in `a` are HOST pointers
+ * (pinned memory gives asynchronous copies); gamma, cu_seqlens, slots and the workspace stay
+ * device pointers.  `staging` is caller-owned device memory of at least
+ * dsla_*_staging_bytes(a); inputs are copied into it, the kernels run on it, and o is copied back,
+ * all on `cuda_stream`.  The caller synchronises the stream before reading o.
+ * ------------------------------------------------------------------------------------------ */
+size_t dsla_prefill_staging_bytes(const dsla_prefill_args* a);
+dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* staging,
+                              size_t staging_bytes, void* cuda_stream);
+size_t dsla_decode_staging_bytes(const dsla_decode_args* a);
+dsla_status dsla_decode_step_host(const dsla_decode_args* a, dsla_state* st, void* staging,
+                                  size_t staging_bytes, void* cuda_stream);
+
+/* Static, human-readable name of a status code. */
+const char* dsla_status_string(dsla_status s);
+
+/* Number of kernels this library has launched in this process (for launch accounting). */
+uint64_t dsla_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSLA_H_ */

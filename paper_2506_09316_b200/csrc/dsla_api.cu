@@ -1,0 +1,283 @@
+// C-ABI entry points of libdsla: argument checks, state store management, kernel dispatch.
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <new>
+
+#include "dsla_internal.cuh"
+
+namespace dsla {
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+__global__ void zero_slots_kernel(float* data, const int32_t* slots, int num_slots, size_t slot_elems) {
+    const int s = slots[blockIdx.y];
+    if (s < 0 || s >= num_slots) return;
+    float4* base = reinterpret_cast<float4*>(data + (size_t)s * slot_elems);
+    const size_t n4 = slot_elems / 4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x)
+        base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+}  // namespace dsla
+
+using namespace dsla;
+
+static bool supported_d(int dk, int dv) { return dk == dv && (dk == 64 || dk == 128); }
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+static size_t esize(dsla_dtype dt) { return dt == DSLA_F32 ? 4 : 2; }
+
+extern "C" {
+
+const char* dsla_status_string(dsla_status s) {
+    switch (s) {
+        case DSLA_OK: return "DSLA_OK";
+        case DSLA_ERR_INVALID_ARG: return "DSLA_ERR_INVALID_ARG";
+        case DSLA_ERR_UNSUPPORTED: return "DSLA_ERR_UNSUPPORTED";
+        case DSLA_ERR_CUDA: return "DSLA_ERR_CUDA";
+        case DSLA_ERR_OOM: return "DSLA_ERR_OOM";
+        case DSLA_ERR_TIMEOUT: return "DSLA_ERR_TIMEOUT";
+    }
+    return "DSLA_ERR_UNKNOWN";
+}
+
+uint64_t dsla_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t dsla_state_bytes(int num_slots, int H, int d_k, int d_v) {
+    if (num_slots <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return 0;
+    return (size_t)num_slots * 2 * (size_t)H * (size_t)d_k * (size_t)d_v * sizeof(float);
+}
+
+dsla_status dsla_state_alloc(dsla_state** out, int num_slots, int H, int d_k, int d_v, void* ext_buf, size_t ext_bytes) {
+    if (!out) return DSLA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (num_slots <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return DSLA_ERR_INVALID_ARG;
+    if (!supported_d(d_k, d_v)) return DSLA_ERR_UNSUPPORTED;
+    const size_t bytes = dsla_state_bytes(num_slots, H, d_k, d_v);
+    if (ext_buf && (ext_bytes < bytes || !aligned(ext_buf, 256))) return DSLA_ERR_INVALID_ARG;
+    dsla_state* st = new (std::nothrow) dsla_state();
+    if (!st) return DSLA_ERR_OOM;
+    st->num_slots = num_slots; st->H = H; st->d_k = d_k; st->d_v = d_v;
+    st->owns_data = ext_buf ? 0 : 1;
+    st->data = static_cast<float*>(ext_buf);
+    st->status = nullptr;
+    if (cudaGetDevice(&st->device) != cudaSuccess) { delete st; return DSLA_ERR_CUDA; }
+    if (!ext_buf) {
+        cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&st->data), bytes);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            delete st;
+            return e == cudaErrorMemoryAllocation ? DSLA_ERR_OOM : DSLA_ERR_CUDA;
+        }
+    }
+    if (cudaMalloc(reinterpret_cast<void**>(&st->status), 256) != cudaSuccess ||
+        cudaMemset(st->status, 0, 256) != cudaSuccess) {
+        (void)cudaGetLastError();
+        if (st->owns_data) cudaFree(st->data);
+        if (st->status) cudaFree(st->status);
+        delete st;
+        return DSLA_ERR_CUDA;
+    }
+    *out = st;
+    return DSLA_OK;
+}
+
+dsla_status dsla_state_free(dsla_state* st) {
+    if (!st) return DSLA_OK;
+    dsla_status rc = DSLA_OK;
+    if (st->owns_data && st->data && cudaFree(st->data) != cudaSuccess) rc = DSLA_ERR_CUDA;
+    if (st->status && cudaFree(st->status) != cudaSuccess) rc = DSLA_ERR_CUDA;
+    delete st;
+    return rc;
+}
+
+void* dsla_state_data(dsla_state* st) { return st ? st->data : nullptr; }
+
+dsla_status dsla_state_zero(dsla_state* st, const int32_t* slots_dev, int n, void* cuda_stream) {
+    if (!st) return DSLA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t slot_elems = (size_t)2 * st->H * st->d_k * st->d_v;
+    if (!slots_dev) {
+        return cudaMemsetAsync(st->data, 0, slot_elems * sizeof(float) * st->num_slots, s) == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
+    }
+    if (n < 0 || n > 65535) return DSLA_ERR_INVALID_ARG;
+    if (n == 0) return DSLA_OK;
+    zero_slots_kernel<<<dim3(32, n), 256, 0, s>>>(st->data, slots_dev, st->num_slots, slot_elems);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
+}
+
+dsla_status dsla_state_last_error(dsla_state* st) {
+    if (!st) return DSLA_ERR_INVALID_ARG;
+    int host = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return DSLA_ERR_CUDA;
+    if (cudaMemcpy(&host, st->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return DSLA_ERR_CUDA;
+    if (host != 0 && cudaMemset(st->status, 0, sizeof(int)) != cudaSuccess) return DSLA_ERR_CUDA;
+    return host == 0 ? DSLA_OK : DSLA_ERR_TIMEOUT;
+}
+
+// ---- prefill ------------------------------------------------------------------------------
+static dsla_impl resolve_impl(const dsla_prefill_args* a) {
+    if (a->impl == DSLA_IMPL_SIMT || a->impl == DSLA_IMPL_TENSOR) return a->impl;
+    return (a->dtype == DSLA_BF16 && a->d_k == 128 && prefill_tc_available()) ? DSLA_IMPL_TENSOR : DSLA_IMPL_SIMT;
+}
+
+static dsla_status check_prefill_sizes(const dsla_prefill_args* a) {
+    if (!a) return DSLA_ERR_INVALID_ARG;
+    if (a->N < 0 || a->T_total < 0 || a->H <= 0 || a->max_seqlen < 0) return DSLA_ERR_INVALID_ARG;
+    if (a->dtype != DSLA_F32 && a->dtype != DSLA_BF16) return DSLA_ERR_INVALID_ARG;
+    if (a->d_k <= 0 || a->d_v <= 0) return DSLA_ERR_INVALID_ARG;
+    if (!supported_d(a->d_k, a->d_v)) return DSLA_ERR_UNSUPPORTED;
+    if (!a->cu_seqlens) {
+        if (a->T < 0 || (long long)a->N * a->T != a->T_total || a->max_seqlen < a->T) return DSLA_ERR_INVALID_ARG;
+    } else if (a->max_seqlen > a->T_total) {
+        return DSLA_ERR_INVALID_ARG;
+    }
+    if (a->impl != DSLA_IMPL_AUTO && a->impl != DSLA_IMPL_SIMT && a->impl != DSLA_IMPL_TENSOR) return DSLA_ERR_INVALID_ARG;
+    const dsla_impl impl = resolve_impl(a);
+    const int chunk = a->chunk == 0 ? 64 : a->chunk;
+    if (impl == DSLA_IMPL_SIMT) {
+        if (chunk != 16 && chunk != 32 && chunk != 64) return DSLA_ERR_UNSUPPORTED;
+    } else {
+        if (a->dtype != DSLA_BF16 || a->d_k != 128 || chunk != 64 || !prefill_tc_available()) return DSLA_ERR_UNSUPPORTED;
+    }
+    return DSLA_OK;
+}
+
+size_t dsla_prefill_workspace_bytes(const dsla_prefill_args* a) {
+    if (check_prefill_sizes(a) != DSLA_OK) return 0;
+    return resolve_impl(a) == DSLA_IMPL_TENSOR ? prefill_tc_workspace_bytes(a) : 0;
+}
+
+static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cudaStream_t s) {
+    dsla_status rc = check_prefill_sizes(a);
+    if (rc != DSLA_OK) return rc;
+    if (!st) return DSLA_ERR_INVALID_ARG;
+    if (st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
+    if (!a->slots && a->N > st->num_slots) return DSLA_ERR_INVALID_ARG;
+    if (a->N == 0) return DSLA_OK;
+    if (!a->gamma) return DSLA_ERR_INVALID_ARG;
+    if (a->T_total > 0) {
+        if (!a->q || !a->k || !a->v || !a->o || !a->g_hist || !a->g_rec) return DSLA_ERR_INVALID_ARG;
+        if (!aligned(a->q, 16) || !aligned(a->k, 16) || !aligned(a->v, 16) || !aligned(a->o, 16)) return DSLA_ERR_INVALID_ARG;
+        if (!aligned(a->g_hist, 4) || !aligned(a->g_rec, 4)) return DSLA_ERR_INVALID_ARG;
+    }
+    const size_t need = dsla_prefill_workspace_bytes(a);
+    if (need > 0 && (!a->workspace || a->workspace_bytes < need || !aligned(a->workspace, 256))) return DSLA_ERR_INVALID_ARG;
+    if (!(a->scale == a->scale)) return DSLA_ERR_INVALID_ARG;
+
+    PrefillParams p{};
+    p.q = a->q; p.k = a->k; p.v = a->v; p.o = a->o;
+    p.g_hist = a->g_hist; p.g_rec = a->g_rec; p.gamma = a->gamma;
+    p.cu_seqlens = a->cu_seqlens; p.slots = a->slots;
+    p.state = st->data; p.status = st->status;
+    p.N = a->N; p.T = a->T; p.H = a->H; p.num_slots = st->num_slots;
+    const int chunk = a->chunk == 0 ? 64 : a->chunk;
+    p.max_chunks = (a->max_seqlen + chunk - 1) / chunk;
+    p.scale = a->scale; p.use_initial_state = a->use_initial_state ? 1 : 0;
+    if (resolve_impl(a) == DSLA_IMPL_TENSOR) return launch_prefill_tc(p, a, s);
+    return launch_prefill_simt(p, a->d_k, chunk, a->dtype, s);
+}
+
+dsla_status dsla_prefill(const dsla_prefill_args* a, dsla_state* st, void* cuda_stream) {
+    return prefill_device(a, st, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---- decode -------------------------------------------------------------------------------
+static dsla_status check_decode(const dsla_decode_args* a, dsla_state* st) {
+    if (!a || !st) return DSLA_ERR_INVALID_ARG;
+    if (a->B < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0) return DSLA_ERR_INVALID_ARG;
+    if (a->dtype != DSLA_F32 && a->dtype != DSLA_BF16) return DSLA_ERR_INVALID_ARG;
+    if (!supported_d(a->d_k, a->d_v)) return DSLA_ERR_UNSUPPORTED;
+    if (st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
+    if (!a->slots && a->B > st->num_slots) return DSLA_ERR_INVALID_ARG;
+    if (!(a->scale == a->scale)) return DSLA_ERR_INVALID_ARG;
+    return DSLA_OK;
+}
+
+static dsla_status decode_device(const dsla_decode_args* a, dsla_state* st, cudaStream_t s) {
+    dsla_status rc = check_decode(a, st);
+    if (rc != DSLA_OK) return rc;
+    if (a->B == 0) return DSLA_OK;
+    if (!a->q || !a->k || !a->v || !a->o || !a->g_hist || !a->g_rec || !a->gamma) return DSLA_ERR_INVALID_ARG;
+    if (!aligned(a->q, 16) || !aligned(a->k, 16) || !aligned(a->v, 16) || !aligned(a->o, 16)) return DSLA_ERR_INVALID_ARG;
+    DecodeParams p{};
+    p.q = a->q; p.k = a->k; p.v = a->v; p.o = a->o;
+    p.g_hist = a->g_hist; p.g_rec = a->g_rec; p.gamma = a->gamma; p.slots = a->slots;
+    p.state = st->data; p.B = a->B; p.H = a->H; p.num_slots = st->num_slots; p.scale = a->scale;
+    return launch_decode(p, a->d_k, a->dtype, s);
+}
+
+dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cuda_stream) {
+    return decode_device(a, st, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---- host-buffer variants -----------------------------------------------------------------
+static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+size_t dsla_prefill_staging_bytes(const dsla_prefill_args* a) {
+    if (check_prefill_sizes(a) != DSLA_OK) return 0;
+    const size_t t = up256((size_t)a->T_total * a->H * a->d_k * esize(a->dtype));
+    const size_t g = up256((size_t)a->T_total * a->H * sizeof(float));
+    return 4 * t + 2 * g;
+}
+
+dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* staging, size_t staging_bytes, void* cuda_stream) {
+    dsla_status rc = check_prefill_sizes(a);
+    if (rc != DSLA_OK) return rc;
+    if (a->T_total == 0) return prefill_device(a, st, static_cast<cudaStream_t>(cuda_stream));
+    const size_t need = dsla_prefill_staging_bytes(a);
+    if (!staging || staging_bytes < need || !aligned(staging, 256)) return DSLA_ERR_INVALID_ARG;
+    if (!a->q || !a->k || !a->v || !a->o || !a->g_hist || !a->g_rec) return DSLA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t tb = (size_t)a->T_total * a->H * a->d_k * esize(a->dtype), t = up256(tb);
+    const size_t gb = (size_t)a->T_total * a->H * sizeof(float), g = up256(gb);
+    char* base = static_cast<char*>(staging);
+    dsla_prefill_args d = *a;
+    d.q = base; d.k = base + t; d.v = base + 2 * t; d.o = base + 3 * t;
+    d.g_hist = reinterpret_cast<float*>(base + 4 * t);
+    d.g_rec = reinterpret_cast<float*>(base + 4 * t + g);
+    bool ok = cudaMemcpyAsync(const_cast<void*>(d.q), a->q, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<void*>(d.k), a->k, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<void*>(d.v), a->v, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<float*>(d.g_hist), a->g_hist, gb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<float*>(d.g_rec), a->g_rec, gb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return DSLA_ERR_CUDA;
+    rc = prefill_device(&d, st, s);
+    if (rc != DSLA_OK) return rc;
+    return cudaMemcpyAsync(a->o, d.o, tb, cudaMemcpyDeviceToHost, s) == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
+}
+
+size_t dsla_decode_staging_bytes(const dsla_decode_args* a) {
+    if (!a || a->B < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0) return 0;
+    const size_t t = up256((size_t)a->B * a->H * a->d_k * esize(a->dtype));
+    const size_t g = up256((size_t)a->B * a->H * sizeof(float));
+    return 4 * t + 2 * g;
+}
+
+dsla_status dsla_decode_step_host(const dsla_decode_args* a, dsla_state* st, void* staging, size_t staging_bytes, void* cuda_stream) {
+    dsla_status rc = check_decode(a, st);
+    if (rc != DSLA_OK) return rc;
+    if (a->B == 0) return DSLA_OK;
+    const size_t need = dsla_decode_staging_bytes(a);
+    if (!staging || staging_bytes < need || !aligned(staging, 256)) return DSLA_ERR_INVALID_ARG;
+    if (!a->q || !a->k || !a->v || !a->o || !a->g_hist || !a->g_rec) return DSLA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t tb = (size_t)a->B * a->H * a->d_k * esize(a->dtype), t = up256(tb);
+    const size_t gb = (size_t)a->B * a->H * sizeof(float), g = up256(gb);
+    char* base = static_cast<char*>(staging);
+    dsla_decode_args d = *a;
+    d.q = base; d.k = base + t; d.v = base + 2 * t; d.o = base + 3 * t;
+    d.g_hist = reinterpret_cast<float*>(base + 4 * t);
+    d.g_rec = reinterpret_cast<float*>(base + 4 * t + g);
+    bool ok = cudaMemcpyAsync(const_cast<void*>(d.q), a->q, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<void*>(d.k), a->k, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<void*>(d.v), a->v, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<float*>(d.g_hist), a->g_hist, gb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(const_cast<float*>(d.g_rec), a->g_rec, gb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!ok) return DSLA_ERR_CUDA;
+    rc = decode_device(&d, st, s);
+    if (rc != DSLA_OK) return rc;
+    return cudaMemcpyAsync(a->o, d.o, tb, cudaMemcpyDeviceToHost, s) == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
+}
+
+}  // extern "C"

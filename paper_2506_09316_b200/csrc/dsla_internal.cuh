@@ -1,0 +1,61 @@
+// Internal declarations shared by the translation units of libdsla (never installed).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dsla.h"
+
+struct dsla_state {
+    float* data;          // [num_slots][2][H][d_k][d_v]
+    int* status;          // device status word (0 = ok)
+    int num_slots, H, d_k, d_v;
+    int owns_data;
+    int device;
+};
+
+namespace dsla {
+
+// Launch parameters of the prefill kernels (all pointers device).
+struct PrefillParams {
+    const void *q, *k, *v;
+    void* o;
+    const float *g_hist, *g_rec, *gamma;
+    const int32_t* cu_seqlens;  // may be null (dense)
+    const int32_t* slots;       // may be null
+    float* state;               // [num_slots][2][H][D][D]
+    int* status;
+    int N, T, H, num_slots;
+    int max_chunks;             // ceil(max_seqlen / C)
+    float scale;
+    int use_initial_state;
+};
+
+struct DecodeParams {
+    const void *q, *k, *v;
+    void* o;
+    const float *g_hist, *g_rec, *gamma;
+    const int32_t* slots;
+    float* state;
+    int B, H, num_slots;
+    float scale;
+};
+
+void count_launch(int n = 1);
+
+// dsla_decode.cu
+dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStream_t s);
+// dsla_prefill_simt.cu
+dsla_status launch_prefill_simt(const PrefillParams& p, int d, int chunk, dsla_dtype dt, cudaStream_t s);
+// dsla_prefill_tc.cu
+bool prefill_tc_available();
+size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a);
+dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a, cudaStream_t s);
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+}  // namespace dsla

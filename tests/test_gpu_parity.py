@@ -1,0 +1,180 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 CPU checker, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_09316_b200 import inputs as gen
+from util import TOL, gpu_prefill, oracle_prefill, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def check_prefill(inp, *, state0=None, slots=None, num_slots=None, chunk=64, impl="auto", scale=1.0, dense=False,
+                  tol=None):
+    tol = tol or TOL[inp.dtype]
+    o, S = gpu_prefill(inp, state0=state0, slots=slots, num_slots=num_slots, chunk=chunk, impl=impl, scale=scale,
+                       dense=dense)
+    o_ref, S_ref = oracle_prefill(inp, state0=state0, slots=slots, scale=scale)
+    lens = inp.seqlens
+    sl = list(range(inp.N)) if slots is None else list(slots)
+    eo = rel_err(o, o_ref)
+    assert eo <= tol, f"o rel err {eo:.3e} > {tol}"
+    for n, L in enumerate(lens):
+        if L == 0 and state0 is None:
+            assert not np.any(S[sl[n]])
+            continue
+        for i in range(2):
+            e = rel_err(S[sl[n], i], S_ref[sl[n], i])
+            assert e <= tol, f"state {i} of sequence {n} rel err {e:.3e} > {tol}"
+    if state0 is not None:   # slots no sequence uses stay as they were
+        untouched = [s for s in range(S.shape[0]) if s not in sl]
+        assert np.array_equal(S[untouched], np.asarray(state0, dtype=np.float32).astype(np.float64)[untouched])
+    return eo
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 131, 513])
+def test_prefill_lengths(dtype, d, T):
+    H = 3 if T < 200 else 1
+    check_prefill(gen.make_dense(7000 + T + d, 1, T, H, d, dtype), impl="simt")
+
+
+@pytest.mark.parametrize("chunk", [16, 32, 64])
+def test_prefill_chunk_invariance(chunk):
+    inp = gen.make_dense(7100, 2, 150, 2, 64, torch.float32)
+    check_prefill(inp, chunk=chunk, impl="simt", dense=True)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_prefill_ragged_with_slots_and_initial_state(dtype):
+    lens = [5, 1, 0, 130, 67]
+    inp = gen.make_packed(7200, lens, 3, 128, dtype)
+    check_prefill(inp, impl="simt")
+    slots = [4, 2, 0, 6, 3]
+    st0 = gen.make_states(7201, 7, 3, 128, 128, std=0.5).numpy()
+    check_prefill(inp, state0=st0, slots=slots, num_slots=7, impl="simt", scale=0.5)
+
+
+def _with_gates(inp, g1, g2, gamma=None):
+    inp.g_hist = torch.as_tensor(np.broadcast_to(g1, inp.g_hist.shape).copy(), dtype=torch.float32)
+    inp.g_rec = torch.as_tensor(np.broadcast_to(g2, inp.g_rec.shape).copy(), dtype=torch.float32)
+    if gamma is not None:
+        inp.gamma = torch.as_tensor(np.asarray(gamma), dtype=torch.float32)
+    return inp
+
+
+@pytest.mark.parametrize("pattern", ["ones", "zeros", "single_zero", "alternating", "swapped", "tiny"])
+def test_prefill_gate_patterns(pattern):
+    T, H, d = 150, 2, 64
+    inp = gen.make_dense(7300, 1, T, H, d, torch.float32)
+    t = np.arange(T)[:, None]
+    if pattern == "ones":
+        _with_gates(inp, 1.0, 1.0)
+    elif pattern == "zeros":
+        _with_gates(inp, 0.0, 0.0)
+    elif pattern == "single_zero":
+        g1 = inp.g_hist.numpy().copy(); g1[70] = 0.0
+        _with_gates(inp, g1, inp.g_rec.numpy())
+    elif pattern == "alternating":
+        _with_gates(inp, np.where(t % 2 == 0, 1.0, 0.5), np.where(t % 2 == 0, 0.5, 1.0))
+    elif pattern == "swapped":
+        _with_gates(inp, inp.g_rec.numpy().copy(), inp.g_hist.numpy().copy())
+    elif pattern == "tiny":
+        _with_gates(inp, 1e-3, np.where(t % 7 == 0, 0.0, 1e-2))
+    st0 = gen.make_states(7301, 1, H, d, d, std=0.3).numpy()
+    check_prefill(inp, impl="simt")
+    check_prefill(inp, state0=st0, impl="simt")
+
+
+@pytest.mark.parametrize("gamma", [0.0, 1.0, 0.5, -0.3, 1.7])
+def test_prefill_gamma_values(gamma):
+    inp = gen.make_dense(7400, 1, 100, 2, 64, torch.float32)
+    inp.gamma = torch.full((2,), gamma, dtype=torch.float32)
+    check_prefill(inp, impl="simt")
+
+
+def run_decode_sequence(dtype, B, H, d, steps, seed, slots=None, num_slots=None, scale=1.0, state_std=0.02):
+    import paper_2506_09316_b200 as dsla
+    from oracle import dsla_oracle as orc
+    num_slots = num_slots or B
+    st0 = gen.make_states(seed, num_slots, H, d, d, std=state_std)
+    st = dsla.dsla_state_alloc(num_slots, H, d, d)
+    st.tensor.copy_(st0)
+    S_ref = st0.double().numpy().copy()
+    sl_dev = None if slots is None else torch.as_tensor(np.asarray(slots), dtype=torch.int32, device="cuda")
+    sl_np = None if slots is None else np.asarray(slots, dtype=np.int32)
+    worst = 0.0
+    for s in range(steps):
+        inp = gen.make_dense(seed + 1 + s, B, 1, H, d, dtype)
+        dv = inp.to("cuda")
+        o = dsla.dsla_decode_step(dv.q, dv.k, dv.v, dv.g_hist, dv.g_rec, dv.gamma, st, slots=sl_dev, scale=scale)
+        f = inp.as_f64()
+        # gamma is drawn per step by the generator; both sides use this step's values
+        o_ref = orc.decode_step(f["q"], f["k"], f["v"], f["g_hist"], f["g_rec"], f["gamma"], S_ref, sl_np, scale=scale)
+        worst = max(worst, rel_err(o.double().cpu().numpy(), o_ref))
+    torch.cuda.synchronize()
+    S = st.tensor.double().cpu().numpy()
+    return worst, max(rel_err(S[:, 0], S_ref[:, 0]), rel_err(S[:, 1], S_ref[:, 1])), S, S_ref
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [64, 128])
+def test_decode_steps(dtype, d):
+    eo, es, _, _ = run_decode_sequence(dtype, 5, 3, d, 12, 7500 + d, state_std=0.05)
+    assert eo <= TOL[dtype] and es <= TOL[dtype], (eo, es)
+
+
+def test_decode_slots_skip_and_repeat():
+    slots = [5, -1, 0, 3]
+    eo, es, S, S_ref = run_decode_sequence(torch.float32, 4, 2, 64, 6, 7600, slots=slots, num_slots=7, scale=0.7)
+    assert eo <= 1e-4 and es <= 1e-4
+    st0 = gen.make_states(7600, 7, 2, 64, 64).double().numpy()
+    assert np.array_equal(S[[1, 2, 4, 6]], st0[[1, 2, 4, 6]])     # untouched slots are bit-identical
+
+
+def test_cfg1_prefill_then_decode():
+    """Workload 1: fp32, B=1 H=4 d=64, 512-token prefill followed by 64 decode steps."""
+    import paper_2506_09316_b200 as dsla
+    from oracle import dsla_oracle as orc
+    c = gen.CONFIGS["cfg1"]
+    T, n_dec = c["T"], c["decode_steps"]
+    inp = gen.make_dense(c["seed"], 1, T + n_dec, c["H"], c["d"], torch.float32)
+    f = inp.as_f64()
+    o_ref, S_ref = orc.prefill(f["q"], f["k"], f["v"], f["g_hist"], f["g_rec"], f["gamma"])
+    dv = inp.to("cuda")
+    st = dsla.dsla_state_alloc(1, c["H"], c["d"], c["d"])
+    o = torch.empty_like(dv.v)
+    dsla.dsla_prefill(dv.q[:T], dv.k[:T], dv.v[:T], dv.g_hist[:T], dv.g_rec[:T], dv.gamma, st, o=o[:T], max_seqlen=T)
+    for t in range(T, T + n_dec):
+        dsla.dsla_decode_step(dv.q[t:t + 1], dv.k[t:t + 1], dv.v[t:t + 1], dv.g_hist[t:t + 1], dv.g_rec[t:t + 1],
+                              dv.gamma, st, o=o[t:t + 1])
+    torch.cuda.synchronize()
+    S = st.tensor.double().cpu().numpy()
+    assert rel_err(o.double().cpu().numpy(), o_ref) <= 1e-4
+    assert rel_err(S[0, 0], S_ref[0, 0]) <= 1e-4 and rel_err(S[0, 1], S_ref[0, 1]) <= 1e-4
+
+
+def test_cfg2_prefill_full():
+    """Workload 2: bf16, B=1 H=32 d=128 T=4096, chunk 64; every output and both final states."""
+    c = gen.CONFIGS["cfg2"]
+    inp = gen.make_dense(c["seed"], 1, c["T"], c["H"], c["d"], torch.bfloat16)
+    e = check_prefill(inp, dense=True)
+    print(f"cfg2 o rel err {e:.3e}")
+
+
+def test_prefill_composition_on_gpu():
+    """prefill(T1) then prefill(T2 | state) equals prefill(T1+T2) (resume from a stored state)."""
+    import paper_2506_09316_b200 as dsla
+    inp = gen.make_dense(7700, 1, 200, 2, 128, torch.bfloat16)
+    o_ref, S_ref = oracle_prefill(inp)
+    dv = inp.to("cuda")
+    st = dsla.dsla_state_alloc(1, 2, 128, 128)
+    o = torch.empty_like(dv.v)
+    a, b = slice(0, 77), slice(77, 200)
+    dsla.dsla_prefill(dv.q[a], dv.k[a], dv.v[a], dv.g_hist[a], dv.g_rec[a], dv.gamma, st, o=o[a], max_seqlen=77)
+    dsla.dsla_prefill(dv.q[b], dv.k[b], dv.v[b], dv.g_hist[b], dv.g_rec[b], dv.gamma, st, o=o[b], max_seqlen=123,
+                      use_initial_state=True)
+    torch.cuda.synchronize()
+    assert rel_err(o.double().cpu().numpy(), o_ref) <= 2e-2
+    assert rel_err(st.tensor[0, 0].double().cpu().numpy(), S_ref[0, 0]) <= 2e-2
