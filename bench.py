@@ -1,0 +1,402 @@
+#!/usr/bin/env python3
+"""Benchmark of the DSLA hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: the chunkwise
+prefill of the prompt(s) followed by one decode step on the states the prefill produced.  The
+default workload is the Llama2-7B-shaped layer (B=1, H=32, d=128, T=4096, bf16, chunk 64).  A
+second section times the batched-decode workload (B=128, H=32, d=128, 32 independent layers,
+256 steps) because decode tokens/s is the other half of the metric.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg5] [--impl ours|reference]
+
+With N > 1 (under torchrun) every rank runs the same per-GPU workload on its own GPU: sequences
+and layers are independent, so there is no data-path collective (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2506_09316_b200 import inputs as gen  # noqa: E402
+
+FLOP_PER_TOKEN_HEAD = lambda d, C: 2 * C * (d + d) + 8 * d * d          # QK^T, PV, 2x QS, 2x K^T V (full squares)
+PREFILL_BYTES_PER_TOKEN_HEAD = lambda d, es: 4 * d * es + 8             # q, k, v, o + two fp32 gates
+DECODE_BYTES_PER_ROW_HEAD = lambda d, es: 4 * d * d * 4 + 4 * d * es + 8  # 2 states read+write, q k v o, gates
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm_gbs=j["hbm_gbs"], bf16_tflops=j["bf16_tflops"],
+                    bf16_tflops_sustained=j.get("bf16_tflops_sustained", j["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _once(self):
+        nv = self.nv
+        self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+            else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+        for bit, name in names.items():
+            if r & bit:
+                self.reasons.add(name)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._once()
+            except Exception:
+                break
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+
+    def stop(self):
+        if self._t:
+            self._stop.set()
+            self._t.join()
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def visible_nvml_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    return rank, world, local
+
+
+def max_over_ranks(x, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def workload_spec(name):
+    c = dict(gen.CONFIGS[name])
+    if name in ("cfg2", "cfg3"):
+        c["lens"] = [c["T"]] * c["B"]
+    elif name == "cfg5":
+        c["lens"] = gen.ragged_lengths(c["seed"], c["N"], c["lo"], c["hi"])
+    else:
+        raise SystemExit(f"workload {name} is not a prefill workload (cfg4 is always reported under 'decode')")
+    return c
+
+
+# --------------------------------------------------------------------------------------------
+def bench_ours(args):
+    import paper_2506_09316_b200 as dsla
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    spec = workload_spec(args.workload)
+    H, d, lens = spec["H"], spec["d"], spec["lens"]
+    N, T_total, max_len = len(lens), int(sum(lens)), int(max(lens))
+    dense = len(set(lens)) == 1
+    bytes_per_set = T_total * H * PREFILL_BYTES_PER_TOKEN_HEAD(d, 2)
+    n_sets = 1 if bytes_per_set > 4 * 126e6 else max(2, int(np.ceil(4 * 126e6 / bytes_per_set)))
+    sets = [gen.make_packed_device(spec["seed"] + 17 * i + 1000 * rank, lens, H, d, torch.bfloat16, device=dev)
+            for i in range(n_sets)]
+    outs = [torch.empty_like(s.v) for s in sets]
+    st = dsla.dsla_state_alloc(N, H, d, d, device=dev)
+    ws_bytes = dsla.binding.dsla_prefill_workspace_bytes(T_total, N, max_len, H, d, torch.bfloat16, 64, args.kernel,
+                                                        dense_T=max_len if dense else None)
+    ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device=dev) if ws_bytes else None
+    # decode inputs for the step's decode leg: one token per sequence
+    dec = gen.make_packed_device(spec["seed"] + 5, [1] * N, H, d, torch.bfloat16, device=dev)
+    dec_o = torch.empty_like(dec.v)
+    stream = torch.cuda.current_stream()
+
+    def step(i, ev=None):
+        s = sets[i % n_sets]
+        if ev:
+            ev[0].record(stream)
+        dsla.dsla_prefill(s.q, s.k, s.v, s.g_hist, s.g_rec, s.gamma, st, o=outs[i % n_sets],
+                          cu_seqlens=None if dense else s.cu_seqlens, max_seqlen=max_len, chunk=64,
+                          impl=args.kernel, workspace=ws)
+        if ev:
+            ev[1].record(stream)
+        dsla.dsla_decode_step(dec.q, dec.k, dec.v, dec.g_hist, dec.g_rec, s.gamma, st, o=dec_o)
+        if ev:
+            ev[2].record(stream)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(visible_nvml_index(local))
+    barrier(world)
+    torch.cuda.synchronize()
+    launches0 = dsla.dsla_launch_count()
+    sampler.start()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_stop = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(i, evs[i])
+    t_stop.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    barrier(world)
+    launches = dsla.dsla_launch_count() - launches0
+    total_ms = max_over_ranks(t_start.elapsed_time(t_stop), world, dev)
+    prefill_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    decode_leg_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    ms_per_step = total_ms / args.steps
+    tokens_per_step = T_total + N
+    value = world * tokens_per_step / (ms_per_step * 1e-3)
+
+    flops = T_total * H * FLOP_PER_TOKEN_HEAD(d, 64)
+    achieved_tf = flops / (prefill_ms * 1e-3) / 1e12
+    roofline = {"kernel": "prefill", "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"], "traffic": None,
+                "peak_source": f"{peaks['source']} burst bf16 (kernel timed alone between events)",
+                "hbm_gbs": bytes_per_set / (prefill_ms * 1e-3) / 1e9,
+                "hbm_frac": bytes_per_set / (prefill_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    # ---- end to end through the host-buffer entry points (pinned host memory)
+    e2e = None
+    if not args.no_e2e:
+        e2e = bench_e2e(dsla, sets[0], dec, st, ws, lens, dense, max_len, args, world, dev)
+
+    decode = None
+    if not args.no_decode:
+        decode = bench_decode(dsla, args, peaks, world, dev, rank)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu_baseline = time_oracle_sample(spec, lens, budget_s=args.cpu_seconds)
+
+    if rank == 0:
+        line = {
+            "metric": "dsla_prefill_plus_decode_tokens_per_s", "value": value, "unit": "tokens/s (one layer)",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: DSLA layer prefill B={N} H={H} d={d} T={lens[0] if dense else 'ragged'} "
+                                   f"(T_total={T_total}) bf16 chunk=64 + 1 decode token per sequence",
+                       "kernel": args.kernel, "l2": f"rotating {n_sets} input sets ({n_sets * bytes_per_set / 1e6:.0f} MB > 126 MB L2)",
+                       "parallelism": f"replicated x{world} (independent sequences, no collective)"},
+            "prefill_only": {"value": world * T_total / (prefill_ms * 1e-3), "unit": "tokens/s (one layer)", "ms": prefill_ms},
+            "decode_leg_ms": decode_leg_ms,
+            "roofline": roofline, "decode": decode, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def bench_e2e(dsla, s, dec, st, ws, lens, dense, max_len, args, world, dev):
+    H, d = s.H, s.d
+    N, T_total = len(lens), int(sum(lens))
+    pin = lambda t: t.cpu().pin_memory()
+    hq, hk, hv, hg1, hg2 = pin(s.q), pin(s.k), pin(s.v), pin(s.g_hist), pin(s.g_rec)
+    ho = torch.empty_like(hv).pin_memory()
+    dq, dk, dv_, dg1, dg2 = pin(dec.q), pin(dec.k), pin(dec.v), pin(dec.g_hist), pin(dec.g_rec)
+    do = torch.empty_like(dv_).pin_memory()
+    stg = torch.empty(dsla.dsla_prefill_staging_bytes(T_total, N, max_len, H, d, torch.bfloat16,
+                                                      dense_T=max_len if dense else None), dtype=torch.uint8, device=dev)
+    stg2 = torch.empty(dsla.dsla_decode_staging_bytes(N, H, d, torch.bfloat16), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        dsla.dsla_prefill_host(hq, hk, hv, hg1, hg2, s.gamma, st, ho, stg, cu_seqlens=None if dense else s.cu_seqlens,
+                               max_seqlen=max_len, chunk=64, impl=args.kernel, workspace=ws)
+        dsla.dsla_decode_step_host(dq, dk, dv_, dg1, dg2, s.gamma, st, do, stg2)
+        stream.synchronize()          # the caller reads o here
+
+    n = max(3, min(args.steps, 10))
+    for _ in range(2):
+        step()
+    barrier(world)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n):
+        step()
+    torch.cuda.synchronize()
+    dt = max_over_ranks(time.perf_counter() - t0, world, dev)
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hg1, hg2, dq, dk, dv_, dg1, dg2))
+    d2h = sum(t.numel() * t.element_size() for t in (ho, do))
+    return {"value": world * (T_total + N) * n / dt, "unit": "tokens/s (one layer)", "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "steps": n, "ms_per_step": dt / n * 1e3,
+            "api": "dsla_prefill_host + dsla_decode_step_host, pinned host buffers, stream sync per step"}
+
+
+def bench_decode(dsla, args, peaks, world, dev, rank):
+    """Batched decode: B=128, H=32, d=128, 32 independent layers, fp32 dual states (17.2 GB)."""
+    c = gen.CONFIGS["cfg4"]
+    B, H, d, L, R = c["B"], c["H"], c["d"], args.decode_layers or c["layers"], c["ring"]
+    steps, warm = args.decode_steps, 3
+    states = [dsla.dsla_state_alloc(B, H, d, d, device=dev) for _ in range(L)]
+    g = torch.Generator(device=dev)
+    g.manual_seed(c["seed"] + rank)
+    for s in states:
+        s.tensor.normal_(0.0, c["state_std"], generator=g)
+    ring = gen.make_packed_device(c["seed"] + 1 + rank, [1] * (L * R * B), H, d, torch.bfloat16, device=dev)
+    view = lambda t: t.view(L, R, B, *t.shape[1:])
+    q, k, v, g1, g2 = map(view, (ring.q, ring.k, ring.v, ring.g_hist, ring.g_rec))
+    o = torch.empty_like(v)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        r = i % R
+        for l in range(L):
+            dsla.dsla_decode_step(q[l, r], k[l, r], v[l, r], g1[l, r], g2[l, r], ring.gamma, states[l], o=o[l, r])
+
+    for i in range(warm):
+        step(i)
+    barrier(world)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    per_launch_s = ms * 1e-3 / (steps * L)
+    bytes_launch = B * H * DECODE_BYTES_PER_ROW_HEAD(d, 2)
+    gbs = bytes_launch / per_launch_s / 1e9
+    return {"workload": f"cfg4: B={B} H={H} d={d} layers={L} steps={steps} bf16 tokens, fp32 states "
+                        f"({L * B * 2 * H * d * d * 4 / 1e9:.1f} GB >> L2), input ring of {R} steps per layer",
+            "value": world * B * steps / (ms * 1e-3), "unit": f"tokens/s ({L}-layer stack)",
+            "layer_tokens_per_s": world * B * steps * L / (ms * 1e-3), "ms_per_step": ms / steps,
+            "gpu_launches": steps * L,
+            "roofline": {"kernel": "decode", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
+                         "us_per_launch": per_launch_s * 1e6}}
+
+
+# --------------------------------------------------------------------------------------------
+def time_oracle_sample(spec, lens, budget_s=15.0):
+    """Times the CPU checker, as it stands, on a bounded sample of the same workload: the first
+    `heads` heads of the first sequences, all their tokens (units are independent)."""
+    from oracle import dsla_oracle as orc
+    H, d = spec["H"], spec["d"]
+    cores = orc.default_threads()
+    rate_guess = 1.5e4 * cores * (128 * 128) / (d * d)       # (token, head) units per second, refined below
+    order = np.argsort(lens)[::-1]
+    seq = int(order[len(order) // 2]) if len(lens) > 1 else 0    # a median-length sequence
+    L = int(lens[seq])
+    heads = int(max(1, min(H, round(budget_s * rate_guess / L))))
+    heads = max(heads, min(H, cores)) if L * min(H, cores) / rate_guess < 4 * budget_s else heads
+    inp = gen.make_packed(spec["seed"], [L], heads, d, torch.bfloat16)
+    f = inp.as_f64()
+    t0 = time.perf_counter()
+    orc.prefill(f["q"], f["k"], f["v"], f["g_hist"], f["g_rec"], f["gamma"], nthreads=cores)
+    dt = time.perf_counter() - t0
+    return {"value": L * heads / H / dt, "unit": "tokens/s (one layer)", "cores": int(min(cores, heads)), "kind": "oracle",
+            "seconds": dt, "sample": f"{heads} of {H} heads x {L} tokens of one sequence (fp64, token by token); "
+                                     f"layer tokens/s = tokens x heads/{H} / time"}
+
+
+def bench_reference(args):
+    """Reference arm: the fp64 CPU checker, as it stands, on this arm's workload and metric."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    spec = workload_spec(args.workload)
+    lens = spec["lens"]
+    per = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    res = None
+    for _ in range(max(0, args.warmup)):
+        time_oracle_sample(spec, lens, budget_s=per / 4)
+    vals, secs = [], 0.0
+    for _ in range(max(1, args.steps)):
+        res = time_oracle_sample(spec, lens, budget_s=per)
+        vals.append(res["value"])
+        secs += res["seconds"]
+    value = float(np.mean(vals))
+    T_total = int(sum(lens))
+    line = {"impl": "reference", "metric": "dsla_prefill_plus_decode_tokens_per_s", "value": value,
+            "unit": "tokens/s (one layer)", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": (T_total + len(lens)) / value * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: same layer shape; each step is a bounded sample ({res['sample']})"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s (one layer)", "cores": res["cores"], "kind": "oracle",
+                             "sample": res["sample"]},
+            "e2e": {"value": value, "unit": "tokens/s (one layer)", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--decode-steps", type=int, default=256)
+    ap.add_argument("--decode-layers", type=int, default=0, help="layers in the decode section (0 = the workload's 32); "
+                    "smaller stacks exist for profiler captures")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(3, args.warmup) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        bench_reference(args)
+    else:
+        bench_ours(args)
+
+
+if __name__ == "__main__":
+    main()
