@@ -26,20 +26,37 @@ namespace {
 
 constexpr int C = 64;                 // tokens per chunk
 constexpr int D = 128;                // head size
-constexpr int NCOMPUTE = 256;         // warps 0-7
-constexpr int WARP_TMA = 8, WARP_MMA = 9;
-constexpr int NTHREADS = 320;
+// Warp roles of the main kernel: 0 = TMA producer, 1 = MMA issuer, 2..9 = tile warps (gates, decay mask,
+// operand scaling), 10..17 = state warps (state rescale + bf16 copy, outputs, initial/final state).
+// A warp may touch only the 32 TMEM lanes of its quadrant (warp index mod 4).
+constexpr int WARP_TMA = 0, WARP_MMA = 1, TILE_W0 = 2, STATE_W0 = 10;
+constexpr int GATE_W0 = 18;               // warps 18,19: gates, decay mask M, per-token factors
+constexpr int NTHREADS = 20 * 32;
 constexpr int STAGE_BYTES = 5 * 16384;   // [K/K~1][K~2][Q/Q~1][Q~2][V]
 constexpr int OFF_K = 0, OFF_Q = 32768, OFF_V = 65536;
 constexpr int OFF_PT = 2 * STAGE_BYTES;  // P~ double buffer, 8 KB each
-constexpr int SMEM_TILES = 2 * STAGE_BYTES + 2 * 8192;
+constexpr int OFF_MASK = OFF_PT + 2 * 8192;  // decay mask M, fp32 [2][64][MASK_PITCH] (one buffer per chunk parity)
+constexpr int MASK_PITCH = 68;               // floats; 272-byte rows keep 16-byte row accesses conflict-free
+constexpr int MASK_BYTES = 64 * MASK_PITCH * 4;
+constexpr int SMEM_TILES = OFF_MASK + 2 * MASK_BYTES;
 constexpr int SMEM_DYN = SMEM_TILES + 1024;  // + alignment slack
+// summary kernel: 4 stages of [K/K~1][K~2][V]
+constexpr int SUM_STAGES = 4, SUM_STAGE_BYTES = 3 * 16384, SUM_OFF_V = 32768;
+constexpr int SUM_NTHREADS = 320, SUM_NCOMPUTE = 256;
+constexpr int SUM_SMEM_DYN = SUM_STAGES * SUM_STAGE_BYTES + 1024;
 // TMEM columns
 constexpr uint32_t COL_S = 0;      // fp32 S1^T [0,128), S2^T [128,256)
 constexpr uint32_t COL_SB = 256;   // bf16 copies: S1^T [256,320), S2^T [320,384)
 constexpr uint32_t COL_O = 384;    // O^T, 64 columns (tokens)
 constexpr uint32_t COL_P = 448;    // P, 64 columns (lanes 0..63 meaningful)
 constexpr size_t SUMMARY_STRIDE = 2 * D * D * sizeof(float) + 256;  // U (both states) + A[2], padded
+
+#ifdef DSLA_TIMELINE
+__device__ long long* g_timeline = nullptr;   // [role 4][chunk 64][event 8]
+#define TL(role, c, ev) do { if (blockIdx.x == 0 && g_timeline && (c) < 64) g_timeline[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
+#else
+#define TL(role, c, ev) do { } while (0)
+#endif
 
 struct TcParams {
     PrefillParams p;
@@ -48,58 +65,39 @@ struct TcParams {
     int cps;            // chunks per segment
 };
 
-struct GateSmem {
-    float b[2][C];      // cumulative log-gate inside the chunk (zero gates skipped)
-    int zc[2][C];       // zero-gate count, inclusive
-    float rowf[2][C];   // weight_i * e^{b_j}, 0 behind a zero gate
-    float w[2][C];      // e^{b_last - b_s} (main) or decay to the end of the segment (summary)
-    float a[2];         // chunk decay
-    float pad[2];
+// Per-token factors of one chunk, per state.
+struct alignas(16) GateSmem {
+    uint32_t rowf[2][C]; // weight_i * (decay from the chunk start through token j), bf16 in both halves
+    uint32_t w[2][C];    // decay from token s to the end of the chunk (or segment), bf16 in both halves
 };
 
-struct Shared {
-    uint64_t full[2], empty[2], p_full, p_free, ready, o_full, o_free, u_full;
+struct alignas(16) Shared {
+    uint64_t full[4], empty[4], p_full[2], p_free, prep_ready[2], sb_ready, s_ready, o_full[2], o_free, u_full, m_ready[2], m_free[2];
     uint32_t tmem_base;
     int abort_flag;
     GateSmem gs[2];
-    double red_b[2][8];
-    int red_z[2][8];
 };
 
-// Inclusive scan of log-gates over one chunk by warps 0 (history) and 1 (recency); each lane owns two
-// consecutive tokens whose gate values (`g0`, `g1`) were fetched earlier.
-__device__ __forceinline__ void gate_scan(GateSmem& gs, int i, int lane, float g0, float g1) {
-    const bool z0 = !(g0 > 0.f), z1 = !(g1 > 0.f);
-    const double l0 = z0 ? 0.0 : (double)__logf(g0), l1 = z1 ? 0.0 : (double)__logf(g1);
-    double run = l0 + l1;
-    int zrun = (int)z0 + (int)z1;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const double up = __shfl_up_sync(0xffffffffu, run, off);
-        const int zup = __shfl_up_sync(0xffffffffu, zrun, off);
-        if (lane >= off) { run += up; zrun += zup; }
-    }
-    const double excl = run - (l0 + l1);
-    const int zexcl = zrun - ((int)z0 + (int)z1);
-    gs.b[i][2 * lane] = (float)(excl + l0);
-    gs.b[i][2 * lane + 1] = (float)run;
-    gs.zc[i][2 * lane] = zexcl + (int)z0;
-    gs.zc[i][2 * lane + 1] = zrun;
+// f rounded to bf16, duplicated into both halves of a 32-bit word
+__device__ __forceinline__ uint32_t dup_bf16(float f) {
+    const uint32_t h = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(f));
+    return h | (h << 16);
 }
 
 __device__ __forceinline__ float load_gate(const float* g, int t, int H, int h, bool ok) {
     return ok ? __ldg(g + (size_t)t * H + h) : 1.f;
 }
 
-// Multiplies the eight bf16 of a 16-byte chunk by f.
-__device__ __forceinline__ uint4 scale8(const uint4 x, float f) {
+// Multiplies the eight bf16 of a 16-byte piece by the bf16 factor held in both halves of f.
+__device__ __forceinline__ uint4 scale8(const uint4 x, const uint32_t f) {
     uint4 y;
     const uint32_t* xi = reinterpret_cast<const uint32_t*>(&x);
     uint32_t* yi = reinterpret_cast<uint32_t*>(&y);
+    const __nv_bfloat162 ff = *reinterpret_cast<const __nv_bfloat162*>(&f);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(&xi[e]);
-        yi[e] = pack_bf16(__low2float(v) * f, __high2float(v) * f);
+        const __nv_bfloat162 r = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&xi[e]), ff);
+        yi[e] = *reinterpret_cast<const uint32_t*>(&r);
     }
     return y;
 }
@@ -126,7 +124,7 @@ __device__ __forceinline__ SeqInfo seq_info(const PrefillParams& p, int n, int g
 // ============================================================================================
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const TcParams tp) {
+                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams tp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
     const PrefillParams& p = tp.p;
@@ -147,12 +145,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (sq.c_begin >= sq.c_end) return;
     const int nc = sq.c_end - sq.c_begin;
     const int t0 = sq.t_begin + sq.c_begin * C;   // first token of this segment
+    const int tok0 = sq.c_begin * C;              // its index inside the sequence
 
     if (tid == 0) {
         mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
-        mbar_init(&sh.empty[0], 1); mbar_init(&sh.empty[1], 1);
-        mbar_init(&sh.p_full, 1); mbar_init(&sh.p_free, 4);
-        mbar_init(&sh.ready, 8); mbar_init(&sh.o_full, 1); mbar_init(&sh.o_free, 8); mbar_init(&sh.u_full, 1);
+        mbar_init(&sh.empty[0], 2); mbar_init(&sh.empty[1], 2);   // MMA commit + the tile group's output store
+        mbar_init(&sh.p_full[0], 1); mbar_init(&sh.p_full[1], 1); mbar_init(&sh.p_free, 2);
+        mbar_init(&sh.prep_ready[0], 4); mbar_init(&sh.prep_ready[1], 4); mbar_init(&sh.sb_ready, 8); mbar_init(&sh.s_ready, 8);
+        mbar_init(&sh.o_full[0], 1); mbar_init(&sh.o_full[1], 1); mbar_init(&sh.o_free, 4); mbar_init(&sh.u_full, 1);
+        mbar_init(&sh.m_ready[0], 2); mbar_init(&sh.m_ready[1], 2);
+        mbar_init(&sh.m_free[0], 4); mbar_init(&sh.m_free[1], 4);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -170,6 +172,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             for (int c = 0; c < nc; ++c) {
                 const int s = c & 1;
                 if (c >= 2) mbar_wait(&sh.empty[s], ((c >> 1) & 1) ^ 1, abortp, p.status);
+                TL(0, c, 0);
                 uint8_t* st = tiles + s * STAGE_BYTES;
                 const int t = t0 + c * C;
                 mbar_arrive_expect_tx(&sh.full[s], 6 * 8192);
@@ -179,6 +182,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tma_load_3d(st + OFF_K + 8192, &map_k, &sh.full[s], 64, h, t);
                 tma_load_3d(st + OFF_V, &map_v, &sh.full[s], 0, h, t);
                 tma_load_3d(st + OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
+                if (c + 2 < nc) {   // pull the tile after next into L2 while this one is in flight
+                    const int t2 = t + 2 * C;
+                    tma_prefetch_3d(&map_q, 0, h, t2); tma_prefetch_3d(&map_q, 64, h, t2);
+                    tma_prefetch_3d(&map_k, 0, h, t2); tma_prefetch_3d(&map_k, 64, h, t2);
+                    tma_prefetch_3d(&map_v, 0, h, t2); tma_prefetch_3d(&map_v, 64, h, t2);
+                }
             }
         }
     } else if (warp == WARP_MMA) {
@@ -192,226 +201,372 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             auto issue_p = [&](int c) {
                 const uint32_t st = sa + (c & 1) * STAGE_BYTES;
                 const uint64_t dq = smem_desc_sw128(st + OFF_Q, 16, 1024), dk = smem_desc_sw128(st + OFF_K, 16, 1024);
-#pragma unroll
+#pragma unroll 2
                 for (int kk = 0; kk < 8; ++kk) {
                     const uint64_t off = (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
                     mma_ss(tb + COL_P, dq + off, dk + off, ID_P, kk > 0);
                 }
-                tc_commit(&sh.p_full);
+                tc_commit(&sh.p_full[c & 1]);
             };
             mbar_wait(&sh.full[0], 0, abortp, p.status);
             tc_fence_after();
             issue_p(0);
             for (int c = 0; c < nc; ++c) {
                 const int s = c & 1;
-                if (c + 1 < nc) {
+                // Scores of the next chunk: issued ahead of this chunk's MMAs when its tile has already
+                // landed (they then run while the state warps work), otherwise right after them.
+                bool p_next_done = c + 1 >= nc;
+                if (!p_next_done && mbar_try_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1) && mbar_try_wait(&sh.p_free, c & 1)) {
+                    tc_fence_after();
+                    issue_p(c + 1);
+                    p_next_done = true;
+                }
+                TL(1, c, 0);
+                mbar_wait(&sh.prep_ready[s], (c >> 1) & 1, abortp, p.status);
+                TL(1, c, 1);
+                if (c > 0) mbar_wait(&sh.o_free, (c - 1) & 1, abortp, p.status);
+                TL(1, c, 2);
+                tc_fence_after();
+                const uint32_t st = sa + s * STAGE_BYTES;
+                // O^T = V^T P~^T + S1^T Q~1^T + S2^T Q~2^T ; the first part does not need the states
+                const uint64_t dv = smem_desc_sw128(st + OFF_V, 8192, 1024);
+                const uint64_t dp = smem_desc_sw128(sa + OFF_PT + s * 8192, 16, 1024);
+#pragma unroll 2
+                for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, dv + (uint64_t)(kk * 128), dp + (uint64_t)(kk * 2), ID_OV, kk > 0);
+                mbar_wait(&sh.sb_ready, c & 1, abortp, p.status);
+                TL(1, c, 3);
+                tc_fence_after();
+#pragma unroll 1
+                for (int i = 0; i < 2; ++i) {
+                    const uint64_t dq = smem_desc_sw128(st + OFF_Q + i * 16384, 16, 1024);
+#pragma unroll 2
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
+                        mma_ts(tb + COL_O, tb + COL_SB + 64 * i + 8 * kk, dq + off, ID_OS, 1);
+                    }
+                }
+                tc_commit(&sh.o_full[s]);
+                // S^T += V^T [K~1 | K~2]   (needs the rescaled fp32 states)
+                mbar_wait(&sh.s_ready, c & 1, abortp, p.status);
+                TL(1, c, 4);
+                tc_fence_after();
+                const uint64_t dkk = smem_desc_sw128(st + OFF_K, 8192, 1024);
+#pragma unroll 2
+                for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, 1);
+                tc_commit(&sh.u_full);
+                tc_commit(&sh.empty[s]);
+                TL(1, c, 5);
+                if (!p_next_done) {
                     mbar_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1, abortp, p.status);
                     mbar_wait(&sh.p_free, c & 1, abortp, p.status);
                     tc_fence_after();
                     issue_p(c + 1);
                 }
-                mbar_wait(&sh.ready, c & 1, abortp, p.status);
-                if (c > 0) mbar_wait(&sh.o_free, (c - 1) & 1, abortp, p.status);
-                tc_fence_after();
-                const uint32_t st = sa + s * STAGE_BYTES;
-                // O^T = S1^T Q~1^T + S2^T Q~2^T + V^T P~^T
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const uint64_t dq = smem_desc_sw128(st + OFF_Q + i * 16384, 16, 1024);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint64_t off = (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
-                        mma_ts(tb + COL_O, tb + COL_SB + 64 * i + 8 * kk, dq + off, ID_OS, (i | kk) > 0);
-                    }
-                }
-                const uint64_t dv = smem_desc_sw128(st + OFF_V, 8192, 1024);
-                const uint64_t dp = smem_desc_sw128(sa + OFF_PT + s * 8192, 16, 1024);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, dv + (uint64_t)(kk * 128), dp + (uint64_t)(kk * 2), ID_OV, 1);
-                tc_commit(&sh.o_full);
-                // S^T += V^T [K~1 | K~2]
-                const uint64_t dkk = smem_desc_sw128(st + OFF_K, 8192, 1024);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, 1);
-                tc_commit(&sh.u_full);
-                tc_commit(&sh.empty[s]);
             }
         }
-    } else {
-        // ------------------------------------------------------------------ compute warps 0..7
-        const int q = warp & 3, hi = warp >> 2;          // TMEM lane quadrant, column half / state index
+    } else if (warp < STATE_W0) {
+        // ------------------------------------------------------------------ tile warps 2..9
+        // Two groups of four warps (one per TMEM lane quadrant) take alternate chunks: group 0 (warps 2..5)
+        // the even ones, group 1 (warps 6..9) the odd ones.  Per chunk a group builds P~ = P (.) M, the scaled
+        // copies of Q and K, and later stores the chunk's outputs.
+        const int grp = (warp - TILE_W0) >> 2;
+        const int gt = tid - (TILE_W0 + 4 * grp) * 32;    // 0..127 inside the group
+        const int q = warp & 3;                           // TMEM lane quadrant
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
-        const float gam = p.gamma[h];
-        const float W1 = gam * p.scale, W2 = (1.f - gam) * p.scale;
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
-        // gate prefetch registers (warps 0, 1 only): two tokens per lane
-        const float* gsrc = warp == 0 ? p.g_hist : p.g_rec;
-        float g0 = 1.f, g1 = 1.f;
-        if (warp < 2) {
-            const int j = 2 * lane;
-            g0 = load_gate(gsrc, t0 + j, p.H, h, sq.c_begin * C + j < sq.len);
-            g1 = load_gate(gsrc, t0 + j + 1, p.H, h, sq.c_begin * C + j + 1 < sq.len);
-        }
-        for (int c = 0; c <= nc; ++c) {
-            const int s = c & 1;
+        for (int c = grp; c < nc; c += 2) {
+            const int s = c & 1;                          // == grp: stage, P~ buffer, gate buffer and M buffer
             GateSmem& gs = sh.gs[s];
             uint8_t* st = tiles + s * STAGE_BYTES;
-            if (c < nc) {
-                // ---- a. gates of this chunk; prefetch the next chunk's
-                if (warp < 2) {
-                    gate_scan(gs, warp, lane, g0, g1);
-                    const int j = (c + 1) * C + 2 * lane;
-                    const bool more = c + 1 < nc;
-                    g0 = load_gate(gsrc, t0 + j, p.H, h, more && sq.c_begin * C + j < sq.len);
-                    g1 = load_gate(gsrc, t0 + j + 1, p.H, h, more && sq.c_begin * C + j + 1 < sq.len);
-                }
-                named_bar_sync(1, NCOMPUTE);
-                if (tid < 2 * C) {
-                    const int i = tid / C, j = tid % C;
-                    const float bl = gs.b[i][C - 1], b = gs.b[i][j];
-                    const int zl = gs.zc[i][C - 1], z = gs.zc[i][j];
-                    const int valid = min(C, sq.len - (sq.c_begin + c) * C);
-                    gs.rowf[i][j] = z == 0 ? (i == 0 ? W1 : W2) * __expf(b) : 0.f;
-                    gs.w[i][j] = (j < valid && z == zl) ? __expf(bl - b) : 0.f;   // rows past the sequence end carry no weight
-                    if (j == 0) gs.a[i] = zl == 0 ? __expf(bl) : 0.f;
-                }
-                named_bar_sync(1, NCOMPUTE);
-                // ---- b. mask (warps 0,1,4,5) and operand scaling (warps 2,3,6,7)
-                mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
-                mbar_wait(&sh.p_full, c & 1, abortp, p.status);
-                tc_fence_after();
-                if (q < 2) {
-                    const int j = 32 * q + lane;
-                    uint8_t* pt = tiles + OFF_PT + s * 8192;
-                    uint32_t r[32];
-                    const bool any = 32 * hi <= 32 * q + 31;     // column block not entirely above the diagonal
-                    if (any) { tmem_ld32(lane_addr + COL_P + 32 * hi, r); tc_wait_ld(); }
-                    __syncwarp();
-                    if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
-                    const float b1 = gs.b[0][j], b2 = gs.b[1][j];
-                    const int z1 = gs.zc[0][j], z2 = gs.zc[1][j];
+            const float* Mm = reinterpret_cast<const float*>(tiles + OFF_MASK + s * MASK_BYTES);
+            if (warp == 4 && lane == 0) TL(2, c, 0);
+            mbar_wait(&sh.m_ready[s], (c >> 1) & 1, abortp, p.status);
+            mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
+            mbar_wait(&sh.p_full[s], (c >> 1) & 1, abortp, p.status);   // P ready; the MMA is also done reading raw Q, K
+            tc_fence_after();
+            if (warp == 4 && lane == 0) TL(2, c, 1);
+            if (q < 2) {
+                // ---- P~ rows 32q..32q+31, all 64 columns
+                const int j = 32 * q + lane;
+                uint8_t* pt = tiles + OFF_PT + s * 8192;
+                uint32_t r0[32], r1[32];
+                tmem_ld32(lane_addr + COL_P, r0);
+                if (q == 1) tmem_ld32(lane_addr + COL_P + 32, r1);
+                tc_wait_ld();
+                __syncwarp();
+                if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
+                const float4* mrow = reinterpret_cast<const float4*>(Mm + j * MASK_PITCH);
+                auto half = [&](const uint32_t (&r)[32], int hcol) {   // 32 columns starting at hcol
 #pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int e = 0; e < 8; e += 2) {
-                            float val[2];
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                const int sc = 32 * hi + 8 * m + e + u;
-                                float mk = 0.f;
-                                if (any && sc <= j) {
-                                    const float d1 = gs.zc[0][sc] == z1 ? __expf(b1 - gs.b[0][sc]) : 0.f;
-                                    const float d2 = gs.zc[1][sc] == z2 ? __expf(b2 - gs.b[1][sc]) : 0.f;
-                                    mk = W1 * d1 + W2 * d2;
-                                }
-                                val[u] = (any && sc <= j) ? __uint_as_float(r[8 * m + e + u]) * mk : 0.f;
-                            }
-                            pk[e >> 1] = pack_bf16(val[0], val[1]);
+                    for (int m4 = 0; m4 < 4; ++m4) {
+                        uint32_t pk[4] = {0u, 0u, 0u, 0u};
+                        // columns hcol + 8 m4 .. +7 ; everything right of the row's 16-block is zero
+                        if (hcol + 8 * m4 <= (j | 15)) {
+                            const float4 ma = mrow[hcol / 4 + 2 * m4], mb = mrow[hcol / 4 + 2 * m4 + 1];
+                            const int o = 8 * m4;
+                            pk[0] = pack_bf16(__uint_as_float(r[o + 0]) * ma.x, __uint_as_float(r[o + 1]) * ma.y);
+                            pk[1] = pack_bf16(__uint_as_float(r[o + 2]) * ma.z, __uint_as_float(r[o + 3]) * ma.w);
+                            pk[2] = pack_bf16(__uint_as_float(r[o + 4]) * mb.x, __uint_as_float(r[o + 5]) * mb.y);
+                            pk[3] = pack_bf16(__uint_as_float(r[o + 6]) * mb.z, __uint_as_float(r[o + 7]) * mb.w);
                         }
-                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 * hi + 8 * m)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, hcol + 8 * m4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
+                };
+                half(r0, 0);
+                if (q == 1) {
+                    half(r1, 32);
                 } else {
-                    const int pt_id = (q - 2) * 32 + lane + 64 * hi;   // 0..127
-#pragma unroll 4
-                    for (int m = 0; m < 8; ++m) {
-                        const int idx = pt_id + 128 * m;               // 16-byte chunk inside a 16 KB tile
-                        const int row = (idx >> 3) & 63;
-                        uint4* qp = reinterpret_cast<uint4*>(st + OFF_Q) + idx;
-                        uint4* kp = reinterpret_cast<uint4*>(st + OFF_K) + idx;
-                        const uint4 xq = *qp, xk = *kp;
-                        *qp = scale8(xq, gs.rowf[0][row]);
-                        *(qp + 1024) = scale8(xq, gs.rowf[1][row]);
-                        *kp = scale8(xk, gs.w[0][row]);
-                        *(kp + 1024) = scale8(xk, gs.w[1][row]);
-                    }
+#pragma unroll
+                    for (int m4 = 0; m4 < 4; ++m4)
+                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 + 8 * m4)) = make_uint4(0u, 0u, 0u, 0u);
                 }
-                fence_proxy_async_smem();
             }
-            // ---- c. outputs of the previous chunk
-            if (c > 0) {
-                const int cp = c - 1;
-                mbar_wait(&sh.o_full, cp & 1, abortp, p.status);
-                tc_fence_after();
-                uint32_t r[32];
-                tmem_ld32(lane_addr + COL_O + 32 * hi, r);
+            {
+                // ---- scaled copies: every thread of the group handles eight 16-byte pieces of Q and of K
+#pragma unroll 2
+                for (int m = 0; m < 8; ++m) {
+                    const int idx = gt + 128 * m;             // 16-byte piece inside a 16 KB tile
+                    const int row = (idx >> 3) & 63;
+                    uint4* qp = reinterpret_cast<uint4*>(st + OFF_Q) + idx;
+                    uint4* kp = reinterpret_cast<uint4*>(st + OFF_K) + idx;
+                    const uint4 xq = *qp, xk = *kp;
+                    const uint32_t f0 = gs.rowf[0][row], f1 = gs.rowf[1][row], w0 = gs.w[0][row], w1 = gs.w[1][row];
+                    *qp = scale8(xq, f0);
+                    *(qp + 1024) = scale8(xq, f1);
+                    *kp = scale8(xk, w0);
+                    *(kp + 1024) = scale8(xk, w1);
+                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(&sh.prep_ready[s]); mbar_arrive(&sh.m_free[s]); }
+            if (warp == 4 && lane == 0) TL(2, c, 2);
+            // ---- outputs of this chunk: lanes = d_v, 64 token columns.  The readout is finished, so the stage's
+            // Q~ region is free: the tile is transposed into it as bf16 [token][d_v] (two swizzled boxes) and
+            // written out by one TMA store; a ragged last chunk is stored row by row instead.
+            mbar_wait(&sh.o_full[s], (c >> 1) & 1, abortp, p.status);
+            tc_fence_after();
+            if (warp == 4 && lane == 0) TL(2, c, 3);
+            const int valid = min(C, sq.len - tok0 - c * C);
+            {
+                uint32_t r0[32], r1[32];
+                tmem_ld32(lane_addr + COL_O, r0);
+                tmem_ld32(lane_addr + COL_O + 32, r1);
                 tc_wait_ld();
                 __syncwarp();
                 if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
-                const int valid = min(C, sq.len - (sq.c_begin + cp) * C);
-                __nv_bfloat16* orow = og + ((size_t)(t0 + cp * C + 32 * hi) * p.H + h) * D + 32 * q + lane;
+                if (warp == 4 && lane == 0) TL(2, c, 4);
+                if (valid == C) {
+                    uint8_t* box = st + OFF_Q + (q >> 1) * 8192;          // d_v half of this quadrant
+                    const int vc = (32 * q + lane) & 63;
 #pragma unroll
-                for (int jj = 0; jj < 32; ++jj)
-                    if (32 * hi + jj < valid) orow[(size_t)jj * p.H * D] = __float2bfloat16_rn(__uint_as_float(r[jj]));
-            }
-            if (c == nc) break;
-            // ---- d. state pass: bf16 copy of S_c for the readout, then S <- a_c S for the update
-            {
-                const float a = gs.a[hi];
-                const uint32_t s_addr = lane_addr + COL_S + 128 * hi;
-                const uint32_t sb_addr = lane_addr + COL_SB + 64 * hi;
-                const int v = 32 * q + lane;
-                if (c == 0) {
-                    // initial state of this segment: slot contents (or zero) pushed through the summaries of
-                    // the earlier segments, S <- A_j S + U_j
-                    const float* base = slot1 + (size_t)hi * state_stride;
-                    const float* wsu = tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr;
-#pragma unroll 1
-                    for (int bt = 0; bt < 4; ++bt) {
-                        float acc[32];
-#pragma unroll
-                        for (int k = 0; k < 32; ++k)
-                            acc[k] = p.use_initial_state ? base[(size_t)(32 * bt + k) * D + v] : 0.f;
-                        for (int jg = 0; jg < g; ++jg) {
-                            const float* u = wsu + (size_t)jg * (SUMMARY_STRIDE / 4);
-                            const float A = u[2 * D * D + hi];
-                            const float* uu = u + (size_t)hi * D * D;
-#pragma unroll
-                            for (int k = 0; k < 32; ++k) acc[k] = fmaf(A, acc[k], uu[(size_t)(32 * bt + k) * D + v]);
-                        }
-                        uint32_t pk[16], sc[32];
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(acc[2 * k], acc[2 * k + 1]);
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) sc[k] = __float_as_uint(acc[k] * a);
-                        tmem_st16(sb_addr + 16 * bt, pk);
-                        tmem_st32(s_addr + 32 * bt, sc);
+                    for (int jj = 0; jj < 32; ++jj) {
+                        *reinterpret_cast<__nv_bfloat16*>(box + sw128_offset(jj, vc)) = __float2bfloat16_rn(__uint_as_float(r0[jj]));
+                        *reinterpret_cast<__nv_bfloat16*>(box + sw128_offset(32 + jj, vc)) = __float2bfloat16_rn(__uint_as_float(r1[jj]));
                     }
+                    fence_proxy_async_smem();
                 } else {
-                    mbar_wait(&sh.u_full, (c - 1) & 1, abortp, p.status);
-                    tc_fence_after();
-                    uint32_t r[2][32];
-                    tmem_ld32(s_addr, r[0]);
+                    __nv_bfloat16* orow = og + ((size_t)(t0 + c * C) * p.H + h) * D + 32 * q + lane;
 #pragma unroll
-                    for (int bt = 0; bt < 4; ++bt) {
-                        tc_wait_ld();
-                        if (bt + 1 < 4) tmem_ld32(s_addr + 32 * (bt + 1), r[(bt + 1) & 1]);
-                        uint32_t (&x)[32] = r[bt & 1];
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(__uint_as_float(x[2 * k]), __uint_as_float(x[2 * k + 1]));
-                        tmem_st16(sb_addr + 16 * bt, pk);
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) x[k] = __float_as_uint(__uint_as_float(x[k]) * a);
-                        tmem_st32(s_addr + 32 * bt, x);
+                    for (int jj = 0; jj < 32; ++jj) {
+                        if (jj < valid) orow[(size_t)jj * p.H * D] = __float2bfloat16_rn(__uint_as_float(r0[jj]));
+                        if (32 + jj < valid) orow[(size_t)(32 + jj) * p.H * D] = __float2bfloat16_rn(__uint_as_float(r1[jj]));
                     }
+                }
+            }
+            named_bar_sync(3 + grp, 128);
+            if (gt == 0) {
+                if (valid == C) {
+                    tma_store_3d(&map_o, st + OFF_Q, 0, h, t0 + c * C);
+                    tma_store_3d(&map_o, st + OFF_Q + 8192, 64, h, t0 + c * C);
+                    tma_store_commit();
+                    tma_store_wait_read();       // the staging bytes have been read; the stage may be refilled
+                }
+                mbar_arrive(&sh.empty[s]);
+            }
+            if (warp == 4 && lane == 0) TL(2, c, 5);
+        }
+        if (gt == 0) tma_store_wait_all();       // global writes of this group's stores are complete
+    } else if (warp >= GATE_W0) {
+        // ------------------------------------------------------------------ gate warps 18,19
+        // Thread s owns token column s of the chunk.  One pass over the rows j multiplies gates together:
+        // d_i(j, s) = prod_{t = s+1..j} g^i_t (exact products: a zero gate gives an exact zero, no logs), so
+        //   M[j][s]   = W1 d_1 + W2 d_2                      (decay mask, 0 above the diagonal)
+        // and the per-token factors come from warp-wide prefix / suffix products:
+        //   w^i_s     = prod_{t > s} g^i_t                    (decay to the end of the chunk)
+        //   rowf^i_j  = W_i prod_{t <= j} g^i_t               (decay from the chunk start through token j)
+        const int sc = tid - GATE_W0 * 32;                // 0..63
+        const float gam = p.gamma[h];
+        const float W1 = gam * p.scale, W2 = (1.f - gam) * p.scale;
+        // each warp keeps all 64 gate pairs of the chunk in registers: lane l holds tokens l and l + 32
+        auto fetch = [&](int c, float2& lo, float2& hi2) {
+            const int j = c * C + lane;
+            const bool in = c < nc;
+            lo.x = fmaxf(load_gate(p.g_hist, t0 + j, p.H, h, in && tok0 + j < sq.len), 0.f);
+            lo.y = fmaxf(load_gate(p.g_rec, t0 + j, p.H, h, in && tok0 + j < sq.len), 0.f);
+            hi2.x = fmaxf(load_gate(p.g_hist, t0 + j + 32, p.H, h, in && tok0 + j + 32 < sq.len), 0.f);
+            hi2.y = fmaxf(load_gate(p.g_rec, t0 + j + 32, p.H, h, in && tok0 + j + 32 < sq.len), 0.f);
+        };
+        float2 nlo, nhi;
+        fetch(0, nlo, nhi);
+        for (int c = 0; c < nc; ++c) {
+            const int s = c & 1;
+            GateSmem& gs = sh.gs[s];
+            float* Mm = reinterpret_cast<float*>(tiles + OFF_MASK + s * MASK_BYTES);
+            const float2 glo = nlo, ghi = nhi;
+            fetch(c + 1, nlo, nhi);
+            if (c >= 2) mbar_wait(&sh.m_free[s], ((c >> 1) - 1) & 1, abortp, p.status);
+            if (warp == GATE_W0 && lane == 0) TL(0, c, 1);
+            {
+                // per-token factors by warp scans: warp 18 for the history state, warp 19 for the recency state
+                const int i = warp - GATE_W0;
+                const float xl = i == 0 ? glo.x : glo.y, xh = i == 0 ? ghi.x : ghi.y;   // tokens lane, lane + 32
+                const float Wi = i == 0 ? W1 : W2;
+                const float pl = warp_prefix_prod(xl, lane), ph0 = warp_prefix_prod(xh, lane);
+                const float tot_lo = __shfl_sync(0xffffffffu, pl, 31);
+                const float sh_in = warp_suffix_prod(xh, lane), sl_in = warp_suffix_prod(xl, lane);   // inclusive suffixes
+                const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0);
+                // exclusive suffix = inclusive suffix of the next lane (1 for the last token of each half)
+                float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
+                if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
+                const int valid = min(C, sq.len - tok0 - c * C);
+                gs.rowf[i][lane] = dup_bf16(Wi * pl);                       // decay from the chunk start through token j
+                gs.rowf[i][lane + 32] = dup_bf16(Wi * tot_lo * ph0);
+                // rows past the end of the sequence carry no weight in the state update
+                gs.w[i][lane] = dup_bf16(lane < valid ? sl_ex * tot_hi : 0.f);
+                gs.w[i][lane + 32] = dup_bf16(lane + 32 < valid ? sh_ex : 0.f);
+            }
+            float d1 = 1.f, d2 = 1.f;
+            float* mcol = Mm + sc;
+#pragma unroll 8
+            for (int j = 0; j < C; ++j) {
+                const float gx = __shfl_sync(0xffffffffu, j < 32 ? glo.x : ghi.x, j & 31);
+                const float gy = __shfl_sync(0xffffffffu, j < 32 ? glo.y : ghi.y, j & 31);
+                if (j > sc) { d1 *= gx; d2 *= gy; }
+                mcol[j * MASK_PITCH] = j >= sc ? fmaf(W2, d2, W1 * d1) : 0.f;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.m_ready[s]);
+            if (warp == GATE_W0 && lane == 0) TL(0, c, 2);
+        }
+    } else {
+        // ------------------------------------------------------------------ state warps 10..17
+        const int q = warp & 3, hi = (warp - STATE_W0) >> 2;   // TMEM lane quadrant, state index
+        const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
+        const uint32_t s_addr = lane_addr + COL_S + 128 * hi;
+        const uint32_t sb_addr = lane_addr + COL_SB + 64 * hi;
+        const int v = 32 * q + lane;
+        const float* gsrc = hi == 0 ? p.g_hist : p.g_rec;
+        // chunk decay a = prod of this state's gates over the chunk (two tokens per lane), fetched one chunk ahead
+        auto chunk_decay = [&](int c) -> float {
+            const int j = c * C + 2 * lane;
+            const bool in = c < nc;
+            const float ga = load_gate(gsrc, t0 + j, p.H, h, in && tok0 + j < sq.len);
+            const float gb = load_gate(gsrc, t0 + j + 1, p.H, h, in && tok0 + j + 1 < sq.len);
+            float pr = fmaxf(ga, 0.f) * fmaxf(gb, 0.f);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) pr *= __shfl_xor_sync(0xffffffffu, pr, off);
+            return pr;
+        };
+        float a_next = chunk_decay(0);
+        for (int c = 0; c < nc; ++c) {
+            const float a = a_next;
+            a_next = chunk_decay(c + 1);
+            if (warp == 12 && lane == 0) TL(3, c, 0);
+            if (c == 0) {
+                // initial state of this segment: slot contents (or zero) pushed through the summaries of
+                // the earlier segments, S <- A_j S + U_j; bf16 copy for the readout, a_0 S for the update
+                const float* base = slot1 + (size_t)hi * state_stride;
+                const float* wsu = tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr;
+#pragma unroll 1
+                for (int bt = 0; bt < 4; ++bt) {
+                    float acc[32];
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        acc[k] = p.use_initial_state ? base[(size_t)(32 * bt + k) * D + v] : 0.f;
+                    for (int jg = 0; jg < g; ++jg) {
+                        const float* u = wsu + (size_t)jg * (SUMMARY_STRIDE / 4);
+                        const float A = u[2 * D * D + hi];
+                        const float* uu = u + (size_t)hi * D * D;
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) acc[k] = fmaf(A, acc[k], uu[(size_t)(32 * bt + k) * D + v]);
+                    }
+                    uint32_t pk[16], sc[32];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(acc[2 * k], acc[2 * k + 1]);
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) sc[k] = __float_as_uint(acc[k] * a);
+                    tmem_st16(sb_addr + 16 * bt, pk);
+                    tmem_st32(s_addr + 32 * bt, sc);
                 }
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.ready);
+                if (lane == 0) { mbar_arrive(&sh.sb_ready); mbar_arrive(&sh.s_ready); }
+                continue;
             }
+            mbar_wait(&sh.u_full, (c - 1) & 1, abortp, p.status);
+            tc_fence_after();
+            if (warp == 12 && lane == 0) TL(3, c, 1);
+            // ---- A. bf16 copy of S_c: the readout of chunk c waits for this
+            {
+                uint32_t r0[32], r1[32];
+                tmem_ld32(s_addr, r0);
+                tmem_ld32(s_addr + 32, r1);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    tc_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(__uint_as_float(r0[2 * k]), __uint_as_float(r0[2 * k + 1]));
+                    tmem_st16(sb_addr + 32 * half, pk);
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(__uint_as_float(r1[2 * k]), __uint_as_float(r1[2 * k + 1]));
+                    tmem_st16(sb_addr + 32 * half + 16, pk);
+                    if (half == 0) { tmem_ld32(s_addr + 64, r0); tmem_ld32(s_addr + 96, r1); }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.sb_ready);
+            }
+            if (warp == 12 && lane == 0) TL(3, c, 2);
+            // ---- B. S <- a_c S: the state update of chunk c waits for this (it runs behind the readout MMAs)
+            {
+                const float2 a2 = make_float2(a, a);
+                uint32_t r0[32], r1[32];
+                tmem_ld32(s_addr, r0);
+                tmem_ld32(s_addr + 32, r1);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    tc_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 32; k += 2) {
+                        const float2 y0 = __fmul2_rn(make_float2(__uint_as_float(r0[k]), __uint_as_float(r0[k + 1])), a2);
+                        const float2 y1 = __fmul2_rn(make_float2(__uint_as_float(r1[k]), __uint_as_float(r1[k + 1])), a2);
+                        r0[k] = __float_as_uint(y0.x); r0[k + 1] = __float_as_uint(y0.y);
+                        r1[k] = __float_as_uint(y1.x); r1[k + 1] = __float_as_uint(y1.y);
+                    }
+                    tmem_st32(s_addr + 64 * half, r0);
+                    tmem_st32(s_addr + 64 * half + 32, r1);
+                    if (half == 0) { tmem_ld32(s_addr + 64, r0); tmem_ld32(s_addr + 96, r1); }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.s_ready);
+            }
+            if (warp == 12 && lane == 0) TL(3, c, 3);
         }
         // ---- final states of this segment's last chunk
         mbar_wait(&sh.u_full, (nc - 1) & 1, abortp, p.status);
         tc_fence_after();
         if (g == sq.last_seg) {
             float* dst = slot1 + (size_t)hi * state_stride;
-            const int v = 32 * q + lane;
 #pragma unroll 1
             for (int bt = 0; bt < 4; ++bt) {
                 uint32_t r[32];
-                tmem_ld32(lane_addr + COL_S + 128 * hi + 32 * bt, r);
+                tmem_ld32(s_addr + 32 * bt, r);
                 tc_wait_ld();
 #pragma unroll
                 for (int k = 0; k < 32; ++k) dst[(size_t)(32 * bt + k) * D + v] = __uint_as_float(r[k]);
@@ -425,10 +580,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
 // ============================================================================================
 // Segment summaries: U_g (both states, from zero) and A_g for every segment but a sequence's last.
-// Weights are taken relative to the END of the segment, so the MMAs accumulate over the whole
-// segment without any rescaling pass.
+// The chunks are walked from the END of the segment backwards while a running product R^i of all
+// later gates is carried, so every token's weight prod_{t > s} g^i_t (to the end of the segment) is a
+// plain product: no logarithms, no rescaling of the accumulator, and a zero gate is exact.
+// Warps 0..7 scale K (warps 0 and 1 first derive the weights), warp 8 drives TMA, warp 9 issues MMAs.
 // ============================================================================================
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(SUM_NTHREADS, 1)
 prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const TcParams tp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
@@ -447,121 +604,98 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     float* out = tp.ws + ((size_t)(n * p.H + h) * tp.nseg + g) * (SUMMARY_STRIDE / 4);
 
     if (tid == 0) {
-        mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
-        mbar_init(&sh.empty[0], 1); mbar_init(&sh.empty[1], 1);
-        mbar_init(&sh.ready, 8); mbar_init(&sh.u_full, 1);
+        for (int s = 0; s < SUM_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.prep_ready[0], 8); mbar_init(&sh.u_full, 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == WARP_MMA) { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
+    if (warp == 9) { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = sh.tmem_base;
     volatile int* abortp = &sh.abort_flag;
 
-    if (warp == WARP_TMA) {
+    // iteration it = 0 .. nc-1 handles chunk nc-1-it
+    if (warp == 8) {
         if (lane == 0) {
             prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-            for (int c = 0; c < nc; ++c) {
-                const int s = c & 1;
-                if (c >= 2) mbar_wait(&sh.empty[s], ((c >> 1) & 1) ^ 1, abortp, p.status);
-                uint8_t* st = tiles + s * STAGE_BYTES;
-                const int t = t0 + c * C;
+            for (int it = 0; it < nc; ++it) {
+                const int s = it % SUM_STAGES, u = it / SUM_STAGES;
+                if (u >= 1) mbar_wait(&sh.empty[s], (u - 1) & 1, abortp, p.status);
+                uint8_t* st = tiles + s * SUM_STAGE_BYTES;
+                const int t = t0 + (nc - 1 - it) * C;
                 mbar_arrive_expect_tx(&sh.full[s], 4 * 8192);
-                tma_load_3d(st + OFF_K, &map_k, &sh.full[s], 0, h, t);
-                tma_load_3d(st + OFF_K + 8192, &map_k, &sh.full[s], 64, h, t);
-                tma_load_3d(st + OFF_V, &map_v, &sh.full[s], 0, h, t);
-                tma_load_3d(st + OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
+                tma_load_3d(st, &map_k, &sh.full[s], 0, h, t);
+                tma_load_3d(st + 8192, &map_k, &sh.full[s], 64, h, t);
+                tma_load_3d(st + SUM_OFF_V, &map_v, &sh.full[s], 0, h, t);
+                tma_load_3d(st + SUM_OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
             }
         }
-    } else if (warp == WARP_MMA) {
+    } else if (warp == 9) {
         if (lane == 0) {
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
-            for (int c = 0; c < nc; ++c) {
-                const int s = c & 1;
-                mbar_wait(&sh.ready, c & 1, abortp, p.status);
+            for (int it = 0; it < nc; ++it) {
+                const int s = it % SUM_STAGES;
+                mbar_wait(&sh.prep_ready[0], it & 1, abortp, p.status);
                 tc_fence_after();
-                const uint32_t st = sa + s * STAGE_BYTES;
-                const uint64_t dv = smem_desc_sw128(st + OFF_V, 8192, 1024), dkk = smem_desc_sw128(st + OFF_K, 8192, 1024);
+                const uint32_t st = sa + s * SUM_STAGE_BYTES;
+                const uint64_t dv = smem_desc_sw128(st + SUM_OFF_V, 8192, 1024), dkk = smem_desc_sw128(st, 8192, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ss(tb, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, (c | kk) > 0);
+                for (int kk = 0; kk < 4; ++kk) mma_ss(tb, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, (it | kk) > 0);
                 tc_commit(&sh.empty[s]);
-                if (c == nc - 1) tc_commit(&sh.u_full);
+                if (it == nc - 1) tc_commit(&sh.u_full);
             }
         }
     } else {
         const int q = warp & 3, hi = warp >> 2;
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
-        // ---- total log-decay and zero-gate count of the whole segment (fp64 sums)
-        double tot[2] = {0.0, 0.0};
-        int ztot[2] = {0, 0};
-        {
-            const int ntok = nc * C;
-            for (int j = tid; j < ntok; j += NCOMPUTE) {
-                const float a = __ldg(p.g_hist + (size_t)(t0 + j) * p.H + h), b = __ldg(p.g_rec + (size_t)(t0 + j) * p.H + h);
-                if (a > 0.f) tot[0] += (double)__logf(a); else ztot[0]++;
-                if (b > 0.f) tot[1] += (double)__logf(b); else ztot[1]++;
-            }
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-                    tot[i] += __shfl_xor_sync(0xffffffffu, tot[i], off);
-                    ztot[i] += __shfl_xor_sync(0xffffffffu, ztot[i], off);
-                }
-                if (lane == 0) { sh.red_b[i][warp] = tot[i]; sh.red_z[i][warp] = ztot[i]; }
-            }
-            named_bar_sync(1, NCOMPUTE);
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                tot[i] = 0.0; ztot[i] = 0;
-                for (int w8 = 0; w8 < 8; ++w8) { tot[i] += sh.red_b[i][w8]; ztot[i] += sh.red_z[i][w8]; }
-            }
-        }
-        double pre[2] = {0.0, 0.0};   // log-decay of the chunks already processed
-        int zpre[2] = {0, 0};
+        // warps 0 / 1: gates of the history / recency state, tokens lane and lane + 32 of the chunk
         const float* gsrc = warp == 0 ? p.g_hist : p.g_rec;
-        float g0 = 1.f, g1 = 1.f;
+        float R = 1.f;                                 // product of the gates of all later chunks
+        float nl = 1.f, nh = 1.f;
         if (warp < 2) {
-            g0 = load_gate(gsrc, t0 + 2 * lane, p.H, h, true);
-            g1 = load_gate(gsrc, t0 + 2 * lane + 1, p.H, h, true);
+            const int t = t0 + (nc - 1) * C + lane;
+            nl = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
+            nh = fmaxf(load_gate(gsrc, t + 32, p.H, h, true), 0.f);
         }
-        for (int c = 0; c < nc; ++c) {
-            const int s = c & 1;
-            GateSmem& gs = sh.gs[s];
-            uint8_t* st = tiles + s * STAGE_BYTES;
+        for (int it = 0; it < nc; ++it) {
+            const int s = it % SUM_STAGES;
+            GateSmem& gs = sh.gs[it & 1];
+            uint8_t* st = tiles + s * SUM_STAGE_BYTES;
             if (warp < 2) {
-                gate_scan(gs, warp, lane, g0, g1);
-                const bool more = c + 1 < nc;
-                const int j = (c + 1) * C + 2 * lane;
-                g0 = load_gate(gsrc, t0 + j, p.H, h, more);
-                g1 = load_gate(gsrc, t0 + j + 1, p.H, h, more);
+                const float xl = nl, xh = nh;
+                if (it + 1 < nc) {
+                    const int t = t0 + (nc - 2 - it) * C + lane;
+                    nl = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
+                    nh = fmaxf(load_gate(gsrc, t + 32, p.H, h, true), 0.f);
+                }
+                const float sh_in = warp_suffix_prod(xh, lane), sl_in = warp_suffix_prod(xl, lane);
+                const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0), tot_lo = __shfl_sync(0xffffffffu, sl_in, 0);
+                float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
+                if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
+                gs.w[warp][lane] = dup_bf16(sl_ex * tot_hi * R);
+                gs.w[warp][lane + 32] = dup_bf16(sh_ex * R);
+                R *= tot_lo * tot_hi;
             }
-            named_bar_sync(1, NCOMPUTE);
-            if (tid < 2 * C) {
-                const int i = tid / C, j = tid % C;
-                const bool open = (ztot[i] - zpre[i] - gs.zc[i][j]) == 0;   // no zero gate after token j
-                gs.w[i][j] = open ? __expf((float)(tot[i] - pre[i] - (double)gs.b[i][j])) : 0.f;
-            }
-            named_bar_sync(1, NCOMPUTE);
+            named_bar_sync(1, SUM_NCOMPUTE);
+            mbar_wait(&sh.full[s], (it / SUM_STAGES) & 1, abortp, p.status);
 #pragma unroll
-            for (int i = 0; i < 2; ++i) { pre[i] += (double)gs.b[i][C - 1]; zpre[i] += gs.zc[i][C - 1]; }
-            mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
-#pragma unroll 4
             for (int m = 0; m < 4; ++m) {
-                const int idx = tid + NCOMPUTE * m;
+                const int idx = tid + SUM_NCOMPUTE * m;
                 const int row = (idx >> 3) & 63;
-                uint4* kp = reinterpret_cast<uint4*>(st + OFF_K) + idx;
+                uint4* kp = reinterpret_cast<uint4*>(st) + idx;
                 const uint4 xk = *kp;
-                *kp = scale8(xk, gs.w[0][row]);
-                *(kp + 1024) = scale8(xk, gs.w[1][row]);
+                const uint32_t w0 = gs.w[0][row], w1 = gs.w[1][row];
+                *kp = scale8(xk, w0);
+                *(kp + 1024) = scale8(xk, w1);
             }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.ready);
+            if (lane == 0) mbar_arrive(&sh.prep_ready[0]);
         }
+        if (warp < 2 && lane == 0) out[2 * D * D + warp] = R;   // A_g: product of every gate of the segment
         mbar_wait(&sh.u_full, 0, abortp, p.status);
         tc_fence_after();
         {
@@ -575,12 +709,11 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 #pragma unroll
                 for (int k = 0; k < 32; ++k) dst[(size_t)(32 * bt + k) * D + v] = __uint_as_float(r[k]);
             }
-            if (tid < 2) out[2 * D * D + tid] = ztot[tid] == 0 ? __expf((float)tot[tid]) : 0.f;
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == WARP_MMA) tmem_dealloc(tb, 256);
+    if (warp == 9) tmem_dealloc(tb, 256);
 }
 
 // ---- host side -------------------------------------------------------------------------------
@@ -632,6 +765,12 @@ void plan(const dsla_prefill_args* a, int* nseg, int* cps) {
 
 }  // namespace
 
+#ifdef DSLA_TIMELINE
+extern "C" int dsla_debug_set_timeline(long long* dev_ptr) {
+    return (int)cudaMemcpyToSymbol(g_timeline, &dev_ptr, sizeof(dev_ptr));
+}
+#endif
+
 bool prefill_tc_available() { return true; }
 
 size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a) {
@@ -650,19 +789,20 @@ dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a
     tp.p = p;
     plan(a, &tp.nseg, &tp.cps);
     tp.ws = tp.nseg > 1 ? static_cast<float*>(a->workspace) : nullptr;
-    CUtensorMap mq, mk, mv;
-    if (!make_map(&mq, p.q, a->T_total, p.H) || !make_map(&mk, p.k, a->T_total, p.H) || !make_map(&mv, p.v, a->T_total, p.H))
+    CUtensorMap mq, mk, mv, mo;
+    if (!make_map(&mq, p.q, a->T_total, p.H) || !make_map(&mk, p.k, a->T_total, p.H) || !make_map(&mv, p.v, a->T_total, p.H) ||
+        !make_map(&mo, p.o, a->T_total, p.H))
         return DSLA_ERR_CUDA;
     if (cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN) != cudaSuccess ||
-        cudaFuncSetAttribute(prefill_tc_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN) != cudaSuccess)
+        cudaFuncSetAttribute(prefill_tc_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SUM_SMEM_DYN) != cudaSuccess)
         return DSLA_ERR_CUDA;
     const long long units = (long long)p.N * p.H;
     if (units * tp.nseg > 0x7fffffffLL) return DSLA_ERR_UNSUPPORTED;
     if (tp.nseg > 1) {
-        prefill_tc_summary_kernel<<<dim3((unsigned)(units * (tp.nseg - 1))), dim3(NTHREADS), SMEM_DYN, s>>>(mk, mv, tp);
+        prefill_tc_summary_kernel<<<dim3((unsigned)(units * (tp.nseg - 1))), dim3(SUM_NTHREADS), SUM_SMEM_DYN, s>>>(mk, mv, tp);
         count_launch();
     }
-    prefill_tc_kernel<<<dim3((unsigned)(units * tp.nseg)), dim3(NTHREADS), SMEM_DYN, s>>>(mq, mk, mv, tp);
+    prefill_tc_kernel<<<dim3((unsigned)(units * tp.nseg)), dim3(NTHREADS), SMEM_DYN, s>>>(mq, mk, mv, mo, tp);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
 }
