@@ -36,7 +36,8 @@ typedef enum {
     DSLA_ERR_UNSUPPORTED = 2, /* head size / chunk / dtype combination that no kernel covers */
     DSLA_ERR_CUDA = 3,        /* a CUDA runtime call failed (no device, launch error, ...) */
     DSLA_ERR_OOM = 4,         /* device allocation failed (dsla_state_alloc only) */
-    DSLA_ERR_TIMEOUT = 5      /* a bounded on-device wait ran out; see dsla_state_last_error */
+    DSLA_ERR_TIMEOUT = 5,     /* a bounded on-device wait ran out; see dsla_state_last_error */
+    DSLA_ERR_SCRATCH_LIMIT = 6 /* dsla_prefill_static_ws only: the call needs more scratch than the built-in array holds */
 } dsla_status;
 
 typedef enum { DSLA_F32 = 0, DSLA_BF16 = 1 } dsla_dtype;
@@ -103,8 +104,8 @@ typedef struct {
     int T_total;                /* rows of q/k/v/o                                               */
     int max_seqlen;             /* upper bound on any sequence length (sizes the grid)           */
     int H, d_k, d_v;
-    int chunk;                  /* C: 16, 32 or 64 for the SIMT kernel; 64 (or 0 = default) for
-                                   the tensor-core kernel, which tiles two chunks per MMA tile   */
+    int chunk;                  /* C: 16, 32 or 64 for the CUDA-core kernel; 64 (or 0 = default) for
+                                   the tensor-core kernel                                        */
     dsla_dtype dtype;           /* dtype of q, k, v, o; the states are always fp32               */
     float scale;                /* multiplies o (1.0f for the plain definition)                  */
     int use_initial_state;      /* 0: start every sequence from zero states; 1: continue from the
@@ -122,6 +123,33 @@ size_t dsla_prefill_workspace_bytes(const dsla_prefill_args* a);
  * length 0 writes no output; its slot is zeroed when use_initial_state == 0 and left as is
  * otherwise.  `a` is a host pointer and is read before the call returns. */
 dsla_status dsla_prefill(const dsla_prefill_args* a, dsla_state* st, void* cuda_stream);
+
+/* Prefill for callers that cannot hand the library a scratch buffer.  (No counterpart in the paper: this
+ * is a deployment convenience, not part of the method.)
+ *
+ * Who needs it: code that runs where device memory cannot be allocated at the time of the call -- for
+ * example a serving loop whose allocator is frozen after start-up, a plug-in that is only handed its
+ * input and output tensors, or a latency-critical path that must never reach cudaMalloc (an allocation
+ * can stall a step for hundreds of milliseconds).  dsla_prefill needs a caller-owned workspace whenever
+ * it splits sequences into segments; this variant uses a fixed array inside the library instead:
+ *
+ *     static __device__ array of DSLA_STATIC_SCRATCH_BYTES bytes, one per GPU that loads the library,
+ *     held until the process exits.
+ *
+ * It computes exactly what dsla_prefill computes for the same arguments (a->workspace and
+ * a->workspace_bytes are ignored) and allocates nothing: no cudaMalloc, no cudaFree, no allocating
+ * library call.  If the arguments would need more scratch than the array holds
+ * (dsla_prefill_workspace_bytes(a) > DSLA_STATIC_SCRATCH_BYTES) nothing is launched and
+ * DSLA_ERR_SCRATCH_LIMIT is returned; use dsla_prefill with your own workspace then.
+ *
+ * The first call on each device looks up the array's device address (one cudaGetSymbolAddress with that
+ * device current); make that first call outside any CUDA stream capture.  Every call on a device shares the
+ * one array and the array keeps whatever the previous call left in it: each call overwrites every entry it
+ * later reads, so nothing has to be cleared, but two calls that overlap on the GPU (different streams,
+ * or different host threads without ordering) race on it.  Run them on one stream or order them with
+ * events. */
+#define DSLA_STATIC_SCRATCH_BYTES (18u << 20)
+dsla_status dsla_prefill_static_ws(const dsla_prefill_args* a, dsla_state* st, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Decode: one step of the recurrence per batch row, fused with the readout and the blend

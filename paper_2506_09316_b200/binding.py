@@ -21,6 +21,8 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 DSLA_OK, DSLA_ERR_INVALID_ARG, DSLA_ERR_UNSUPPORTED, DSLA_ERR_CUDA, DSLA_ERR_OOM, DSLA_ERR_TIMEOUT = range(6)
+DSLA_ERR_SCRATCH_LIMIT = 6
+DSLA_STATIC_SCRATCH_BYTES = 18 << 20
 DSLA_F32, DSLA_BF16 = 0, 1
 DSLA_IMPL_AUTO, DSLA_IMPL_SIMT, DSLA_IMPL_TENSOR = 0, 1, 2
 _DTYPES = {torch.float32: DSLA_F32, torch.bfloat16: DSLA_BF16}
@@ -64,6 +66,8 @@ _lib.dsla_prefill_workspace_bytes.argtypes = [POINTER(dsla_prefill_args)]
 _lib.dsla_prefill_workspace_bytes.restype = c_size_t
 _lib.dsla_prefill.argtypes = [POINTER(dsla_prefill_args), c_void_p, c_void_p]
 _lib.dsla_prefill.restype = c_int
+_lib.dsla_prefill_static_ws.argtypes = [POINTER(dsla_prefill_args), c_void_p, c_void_p]
+_lib.dsla_prefill_static_ws.restype = c_int
 _lib.dsla_decode_step.argtypes = [POINTER(dsla_decode_args), c_void_p, c_void_p]
 _lib.dsla_decode_step.restype = c_int
 _lib.dsla_prefill_staging_bytes.argtypes = [POINTER(dsla_prefill_args)]
@@ -209,6 +213,29 @@ def dsla_prefill(q, k, v, g_hist, g_rec, gamma, st: DslaState, *, o=None, cu_seq
     a = _prefill_args(q, k, v, o, g_hist, g_rec, gamma, cu_seqlens, slots, N, T, max_seqlen, chunk, scale,
                       use_initial_state, impl, workspace)
     _check(_lib.dsla_prefill(byref(a), st.handle, _stream(stream)), "dsla_prefill")
+    return o
+
+
+def dsla_prefill_static_ws(q, k, v, g_hist, g_rec, gamma, st: DslaState, *, o=None, cu_seqlens=None, slots=None,
+                           max_seqlen=None, chunk=64, scale=1.0, use_initial_state=False, impl="auto", stream=None):
+    """Same as ``dsla_prefill`` but the scratch for the segment summaries is the fixed array inside the
+    library, so neither the caller nor the library allocates anything for the call (``o`` must then be
+    passed in by callers that cannot allocate).  Raises DslaError(DSLA_ERR_SCRATCH_LIMIT) when the sizes
+    need more than DSLA_STATIC_SCRATCH_BYTES.  Calls that overlap on the GPU race on the shared array."""
+    T_total = q.shape[0]
+    if cu_seqlens is None:
+        T = int(max_seqlen) if max_seqlen is not None else T_total
+        N = T_total // T if T > 0 else 0
+        max_seqlen = T
+    else:
+        N, T = cu_seqlens.numel() - 1, 0
+        if max_seqlen is None:
+            raise ValueError("max_seqlen is required with cu_seqlens")
+    if o is None:
+        o = torch.empty_like(v)
+    a = _prefill_args(q, k, v, o, g_hist, g_rec, gamma, cu_seqlens, slots, N, T, max_seqlen, chunk, scale,
+                      use_initial_state, impl, None)
+    _check(_lib.dsla_prefill_static_ws(byref(a), st.handle, _stream(stream)), "dsla_prefill_static_ws")
     return o
 
 

@@ -36,6 +36,7 @@ const char* dsla_status_string(dsla_status s) {
         case DSLA_ERR_CUDA: return "DSLA_ERR_CUDA";
         case DSLA_ERR_OOM: return "DSLA_ERR_OOM";
         case DSLA_ERR_TIMEOUT: return "DSLA_ERR_TIMEOUT";
+        case DSLA_ERR_SCRATCH_LIMIT: return "DSLA_ERR_SCRATCH_LIMIT";
     }
     return "DSLA_ERR_UNKNOWN";
 }
@@ -177,6 +178,12 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     if (resolve_impl(a) == DSLA_IMPL_TENSOR) return launch_prefill_tc(p, a, s);
     return launch_prefill_simt(p, a->d_k, chunk, a->dtype, s);
 }
+
+}  // extern "C"
+namespace dsla {
+dsla_status prefill_checked(const dsla_prefill_args* a, dsla_state* st, cudaStream_t s) { return prefill_device(a, st, s); }
+}
+extern "C" {
 
 dsla_status dsla_prefill(const dsla_prefill_args* a, dsla_state* st, void* cuda_stream) {
     return prefill_device(a, st, static_cast<cudaStream_t>(cuda_stream));

@@ -43,6 +43,8 @@ struct DecodeParams {
 
 void count_launch(int n = 1);
 
+// dsla_api.cu: argument checks + dispatch shared by the prefill entry points
+dsla_status prefill_checked(const dsla_prefill_args* a, dsla_state* st, cudaStream_t s);
 // dsla_decode.cu
 dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStream_t s);
 // dsla_prefill_simt.cu
