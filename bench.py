@@ -202,8 +202,11 @@ def bench_ours(args):
 
     flops = T_total * H * FLOP_PER_TOKEN_HEAD(d, 64)
     achieved_tf = flops / (prefill_ms * 1e-3) / 1e12
-    roofline = {"kernel": "prefill", "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"], "traffic": None,
+    # DRAM bytes per prefill from the ncu capture summarised in profiles/prefill_tc_cfg2.md (main + summary kernel)
+    traffic = 182.2e6 if (args.workload == "cfg2" and args.kernel != "simt") else None
+    roofline = {"kernel": "prefill (summary + main launch)", "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"], "traffic": traffic,
+                "algorithmic_bytes": bytes_per_set, "algorithmic_flops": flops,
                 "peak_source": f"{peaks['source']} burst bf16 (kernel timed alone between events)",
                 "hbm_gbs": bytes_per_set / (prefill_ms * 1e-3) / 1e9,
                 "hbm_frac": bytes_per_set / (prefill_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
@@ -318,7 +321,8 @@ def bench_decode(dsla, args, peaks, world, dev, rank):
             "layer_tokens_per_s": world * B * steps * L / (ms * 1e-3), "ms_per_step": ms / steps,
             "gpu_launches": steps * L,
             "roofline": {"kernel": "decode", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peaks['source']} copy bandwidth",
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": 1021.9e6 if B == 128 else None,  # profiles/decode_kernel_cfg4.md
+                         "algorithmic_bytes": bytes_launch, "peak_source": f"{peaks['source']} copy bandwidth",
                          "us_per_launch": per_launch_s * 1e6}}
 
 
