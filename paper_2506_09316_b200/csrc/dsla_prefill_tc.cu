@@ -15,6 +15,8 @@
 // (U_g = sum_s (prod of later gates in the segment) k_s^T v_s and A_g = prod of the segment's
 // gates) into the workspace; the main kernel combines the summaries of earlier segments into its
 // initial state and then runs its segment.
+#include <type_traits>
+
 #include "dsla_internal.cuh"
 #include "tc_utils.cuh"
 
@@ -35,10 +37,11 @@ constexpr int NTHREADS = 20 * 32;
 constexpr int STAGE_BYTES = 5 * 16384;   // [K/K~1][K~2][Q/Q~1][Q~2][V]
 constexpr int OFF_K = 0, OFF_Q = 32768, OFF_V = 65536;
 constexpr int OFF_PT = 2 * STAGE_BYTES;  // P~ double buffer, 8 KB each
-constexpr int OFF_MASK = OFF_PT + 2 * 8192;  // decay mask M, fp32 [2][64][MASK_PITCH] (one buffer per chunk parity)
-constexpr int MASK_PITCH = 68;               // floats; 272-byte rows keep 16-byte row accesses conflict-free
-constexpr int MASK_BYTES = 64 * MASK_PITCH * 4;
-constexpr int SMEM_TILES = OFF_MASK + 2 * MASK_BYTES;
+constexpr int OFF_MASK = OFF_PT + 2 * 8192;  // decay mask M, bf16 [2][64][MASK_PITCH] (one buffer per chunk parity)
+constexpr int MASK_PITCH = 72;               // bf16 elements; 144-byte rows keep 16-byte row accesses conflict-free
+constexpr int MASK_BYTES = 64 * MASK_PITCH * 2;
+constexpr int OFF_OSTG = OFF_MASK + 2 * MASK_BYTES + 1024 - (2 * MASK_BYTES) % 1024;   // output staging, 2 x 8 KB boxes
+constexpr int SMEM_TILES = OFF_OSTG + 16384;
 constexpr int SMEM_DYN = SMEM_TILES + 1024;  // + alignment slack
 // summary kernel: 4 stages of [K/K~1][K~2][V]
 constexpr int SUM_STAGES = 4, SUM_STAGE_BYTES = 3 * 16384, SUM_OFF_V = 32768;
@@ -53,9 +56,12 @@ constexpr size_t SUMMARY_STRIDE = 2 * D * D * sizeof(float) + 256;  // U (both s
 
 #ifdef DSLA_TIMELINE
 __device__ long long* g_timeline = nullptr;   // [role 4][chunk 64][event 8]
-#define TL(role, c, ev) do { if (blockIdx.x == 0 && g_timeline && (c) < 64) g_timeline[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
+__device__ int g_timeline_block = 0;
+#define TL(role, c, ev) do { if (tlp && (c) < 64) tlp[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
+#define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr
 #else
 #define TL(role, c, ev) do { } while (0)
+#define TL_INIT do { } while (0)
 #endif
 
 struct TcParams {
@@ -72,7 +78,7 @@ struct alignas(16) GateSmem {
 };
 
 struct alignas(16) Shared {
-    uint64_t full[4], empty[4], p_full[2], p_free, prep_ready[2], sb_ready, s_ready, o_full[2], o_free, u_full, m_ready[2], m_free[2];
+    uint64_t full[4], empty[4], p_full[2], p_free, prep_ready[2], sb_ready[2], s_ready[2], o_full[2], o_free, u_full[2], m_ready[2], m_free[2], stg_free;
     uint32_t tmem_base;
     int abort_flag;
     GateSmem gs[2];
@@ -119,6 +125,49 @@ __device__ __forceinline__ SeqInfo seq_info(const PrefillParams& p, int n, int g
     return s;
 }
 
+// Initial state of a segment (cold path, kept out of line so the chunk loop stays small): the slot
+// contents (or zero) pushed through the summaries of the earlier segments, S <- A_j S + U_j; writes the bf16
+// copy for the readout and a_0 S for the first update.  One thread = one d_v lane of one state.
+__device__ __noinline__ void init_state_pass(const float* base, int use_initial_state, const float* wsu, int g, int hi, int v,
+                                             float a, uint32_t s_addr, uint32_t sb_addr) {
+#pragma unroll 1
+    for (int bt = 0; bt < 4; ++bt) {
+        float acc[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) acc[k] = use_initial_state ? base[(size_t)(32 * bt + k) * D + v] : 0.f;
+#pragma unroll 1
+        for (int jg = 0; jg < g; ++jg) {
+            const float* u = wsu + (size_t)jg * (SUMMARY_STRIDE / 4);
+            const float A = __ldg(u + 2 * D * D + hi);
+            const float* uu = u + (size_t)hi * D * D;
+            float x[32];
+#pragma unroll
+            for (int k = 0; k < 32; ++k) x[k] = __ldg(uu + (size_t)(32 * bt + k) * D + v);
+#pragma unroll
+            for (int k = 0; k < 32; ++k) acc[k] = fmaf(A, acc[k], x[k]);
+        }
+        uint32_t pk[16], sc[32];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(acc[2 * k], acc[2 * k + 1]);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) sc[k] = __float_as_uint(acc[k] * a);
+        tmem_st16(sb_addr + 16 * bt, pk);
+        tmem_st32(s_addr + 32 * bt, sc);
+    }
+}
+
+// Final fp32 state of one (state, d_v lane) from TMEM to global memory [d_k][d_v] (cold path, out of line).
+__device__ __noinline__ void store_state(float* dst, int v, uint32_t s_addr) {
+#pragma unroll 1
+    for (int bt = 0; bt < 4; ++bt) {
+        uint32_t r[32];
+        tmem_ld32(s_addr + 32 * bt, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) dst[(size_t)(32 * bt + k) * D + v] = __uint_as_float(r[k]);
+    }
+}
+
 // ============================================================================================
 // Main kernel
 // ============================================================================================
@@ -146,15 +195,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int nc = sq.c_end - sq.c_begin;
     const int t0 = sq.t_begin + sq.c_begin * C;   // first token of this segment
     const int tok0 = sq.c_begin * C;              // its index inside the sequence
+    TL_INIT;
+    if (tid == 0) TL(0, 63, 6);
 
     if (tid == 0) {
         mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
-        mbar_init(&sh.empty[0], 2); mbar_init(&sh.empty[1], 2);   // MMA commit + the tile group's output store
-        mbar_init(&sh.p_full[0], 1); mbar_init(&sh.p_full[1], 1); mbar_init(&sh.p_free, 2);
-        mbar_init(&sh.prep_ready[0], 4); mbar_init(&sh.prep_ready[1], 4); mbar_init(&sh.sb_ready, 8); mbar_init(&sh.s_ready, 8);
-        mbar_init(&sh.o_full[0], 1); mbar_init(&sh.o_full[1], 1); mbar_init(&sh.o_free, 4); mbar_init(&sh.u_full, 1);
+        mbar_init(&sh.empty[0], 1); mbar_init(&sh.empty[1], 1);
+        mbar_init(&sh.p_full[0], 1); mbar_init(&sh.p_free, 8);   // every tile warp passes p_full before P is overwritten
+        mbar_init(&sh.prep_ready[0], 8);
+        mbar_init(&sh.sb_ready[0], 4); mbar_init(&sh.sb_ready[1], 4); mbar_init(&sh.s_ready[0], 4); mbar_init(&sh.s_ready[1], 4);
+        mbar_init(&sh.o_full[0], 1); mbar_init(&sh.o_free, 8); mbar_init(&sh.u_full[0], 1); mbar_init(&sh.u_full[1], 1);
         mbar_init(&sh.m_ready[0], 2); mbar_init(&sh.m_ready[1], 2);
-        mbar_init(&sh.m_free[0], 4); mbar_init(&sh.m_free[1], 4);
+        mbar_init(&sh.m_free[0], 8); mbar_init(&sh.m_free[1], 8);
+        mbar_init(&sh.stg_free, 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -182,6 +235,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tma_load_3d(st + OFF_K + 8192, &map_k, &sh.full[s], 64, h, t);
                 tma_load_3d(st + OFF_V, &map_v, &sh.full[s], 0, h, t);
                 tma_load_3d(st + OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
+#ifdef DSLA_TIMELINE
+                mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
+                TL(0, c, 3);
+#endif
                 if (c + 2 < nc) {   // pull the tile after next into L2 while this one is in flight
                     const int t2 = t + 2 * C;
                     tma_prefetch_3d(&map_q, 0, h, t2); tma_prefetch_3d(&map_q, 64, h, t2);
@@ -197,205 +254,230 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OS = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OV = idesc_bf16(128, 64, 1, 0);
-            constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
+            constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
+            // Descriptors of stage 0; stage 1 and the k-steps are reached by adding constants to the address field.
+            constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4), PT_STEP = (uint64_t)(8192 >> 4);
+            const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dk0 = smem_desc_sw128(sa + OFF_K, 16, 1024);
+            const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
+            const uint64_t dp0 = smem_desc_sw128(sa + OFF_PT, 16, 1024);
+            // One thread issues every MMA of the CTA.  Groups of four with compile-time operand steps cost about 45
+            // cycles per issue (a rolled loop about 80), which keeps the issue rate above the tensor pipe's.
+            auto run_ss4 = [&](uint32_t d, uint64_t a, uint64_t b, auto astep, auto bstep, uint32_t idesc, uint32_t acc) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ss(d, a + (uint64_t)(kk * decltype(astep)::value), b + (uint64_t)(kk * decltype(bstep)::value), idesc, kk > 0 ? 1u : acc);
+            };
+            auto run_ts4 = [&](uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_ts(d, a_tmem + 8 * kk, b + (uint64_t)(2 * kk), idesc, 1);
+            };
+            using S2 = std::integral_constant<int, 2>;
+            using S128 = std::integral_constant<int, 128>;
             auto issue_p = [&](int c) {
-                const uint32_t st = sa + (c & 1) * STAGE_BYTES;
-                const uint64_t dq = smem_desc_sw128(st + OFF_Q, 16, 1024), dk = smem_desc_sw128(st + OFF_K, 16, 1024);
-#pragma unroll 2
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
-                    mma_ss(tb + COL_P, dq + off, dk + off, ID_P, kk > 0);
-                }
-                tc_commit(&sh.p_full[c & 1]);
+                const uint64_t so = (uint64_t)(c & 1) * STAGE_STEP;
+                // K-major operands: four 32-byte k-steps inside a 64-element block, then the next block 8 KB further
+#pragma unroll 1
+                for (int blk = 0; blk < 2; ++blk)
+                    run_ss4(tb + COL_P, dq0 + so + (uint64_t)(512 * blk), dk0 + so + (uint64_t)(512 * blk), S2{}, S2{}, ID_P, (uint32_t)blk);
+                tc_commit(&sh.p_full[0]);
             };
             mbar_wait(&sh.full[0], 0, abortp, p.status);
             tc_fence_after();
             issue_p(0);
             for (int c = 0; c < nc; ++c) {
                 const int s = c & 1;
-                // Scores of the next chunk: issued ahead of this chunk's MMAs when its tile has already
-                // landed (they then run while the state warps work), otherwise right after them.
+                const uint64_t so = (uint64_t)s * STAGE_STEP;
+                // Scores of the next chunk go out as soon as its tile has landed and every tile warp has seen P_c:
+                // polled between the MMA groups of this chunk so the tile warps can start on the next one early.
+                // stage: 0 wait operands, 1 V part, 2/3 state parts, 4/5 state updates, 6 done
                 bool p_next_done = c + 1 >= nc;
-                if (!p_next_done && mbar_try_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1) && mbar_try_wait(&sh.p_free, c & 1)) {
-                    tc_fence_after();
-                    issue_p(c + 1);
-                    p_next_done = true;
-                }
-                TL(1, c, 0);
-                mbar_wait(&sh.prep_ready[s], (c >> 1) & 1, abortp, p.status);
-                TL(1, c, 1);
-                if (c > 0) mbar_wait(&sh.o_free, (c - 1) & 1, abortp, p.status);
-                TL(1, c, 2);
-                tc_fence_after();
-                const uint32_t st = sa + s * STAGE_BYTES;
-                // O^T = V^T P~^T + S1^T Q~1^T + S2^T Q~2^T ; the first part does not need the states
-                const uint64_t dv = smem_desc_sw128(st + OFF_V, 8192, 1024);
-                const uint64_t dp = smem_desc_sw128(sa + OFF_PT + s * 8192, 16, 1024);
-#pragma unroll 2
-                for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, dv + (uint64_t)(kk * 128), dp + (uint64_t)(kk * 2), ID_OV, kk > 0);
-                mbar_wait(&sh.sb_ready, c & 1, abortp, p.status);
-                TL(1, c, 3);
-                tc_fence_after();
+                int stage = 0;
 #pragma unroll 1
-                for (int i = 0; i < 2; ++i) {
-                    const uint64_t dq = smem_desc_sw128(st + OFF_Q + i * 16384, 16, 1024);
-#pragma unroll 2
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint64_t off = (uint64_t)(((kk >> 2) * 8192 + (kk & 3) * 32) >> 4);
-                        mma_ts(tb + COL_O, tb + COL_SB + 64 * i + 8 * kk, dq + off, ID_OS, 1);
+                for (uint32_t spin = 0; spin < 40000000u && !(p_next_done && stage == 6); ++spin) {
+                    if (!p_next_done && mbar_test_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1) && mbar_test_wait(&sh.p_free, c & 1)) {
+                        tc_fence_after();
+                        issue_p(c + 1);
+                        p_next_done = true;
+                        TL(1, c + 1, 7);
                     }
+                    if (stage == 0) {
+                        if (mbar_test_wait(&sh.prep_ready[0], c & 1) && (c == 0 || mbar_test_wait(&sh.o_free, (c - 1) & 1))) {
+                            TL(1, c, 1);
+                            tc_fence_after();
+                            // O^T = V^T P~^T + S1^T Q~1^T + S2^T Q~2^T ; the first part does not need the states
+                            run_ss4(tb + COL_O, dv0 + so, dp0 + (uint64_t)s * PT_STEP, S128{}, S2{}, ID_OV, 0);
+                            stage = 2;
+                        }
+                    } else if (stage == 2 || stage == 3) {
+                        // each state has its own hand-offs: the copy / rescale pass of one runs under the MMAs of the other
+                        const int i = stage - 2;
+                        if (mbar_test_wait(&sh.sb_ready[i], c & 1)) {
+                            if (i == 0) TL(1, c, 3);
+                            tc_fence_after();
+                            const uint64_t dq = dq0 + so + (uint64_t)(i * (16384 >> 4));
+                            run_ts4(tb + COL_O, tb + COL_SB + 64 * i, dq, ID_OS);
+                            run_ts4(tb + COL_O, tb + COL_SB + 64 * i + 32, dq + 512, ID_OS);
+                            if (i == 1) { tc_commit(&sh.o_full[0]); TL(1, c, 6); }
+                            ++stage;
+                        }
+                    } else if (stage == 4 || stage == 5) {
+                        // S^i^T += V^T K~i   (needs the rescaled fp32 state i)
+                        const int i = stage - 4;
+                        if (mbar_test_wait(&sh.s_ready[i], c & 1)) {
+                            if (i == 0) TL(1, c, 4);
+                            tc_fence_after();
+                            run_ss4(tb + COL_S + 128 * i, dv0 + so, dkn0 + so + (uint64_t)(i * (16384 >> 4)), S128{}, S128{}, ID_U, 1);
+                            tc_commit(&sh.u_full[i]);
+                            if (i == 1) { tc_commit(&sh.empty[s]); TL(1, c, 5); }
+                            ++stage;
+                        }
+                    }
+                    if ((spin & 4095u) == 4095u && *abortp) break;
                 }
-                tc_commit(&sh.o_full[s]);
-                // S^T += V^T [K~1 | K~2]   (needs the rescaled fp32 states)
-                mbar_wait(&sh.s_ready, c & 1, abortp, p.status);
-                TL(1, c, 4);
-                tc_fence_after();
-                const uint64_t dkk = smem_desc_sw128(st + OFF_K, 8192, 1024);
-#pragma unroll 2
-                for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, 1);
-                tc_commit(&sh.u_full);
-                tc_commit(&sh.empty[s]);
-                TL(1, c, 5);
-                if (!p_next_done) {
-                    mbar_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1, abortp, p.status);
-                    mbar_wait(&sh.p_free, c & 1, abortp, p.status);
-                    tc_fence_after();
-                    issue_p(c + 1);
-                }
+                if (!(p_next_done && stage == 6) && !*abortp) { *abortp = 1; atomicExch(p.status, 5); }
             }
         }
     } else if (warp < STATE_W0) {
         // ------------------------------------------------------------------ tile warps 2..9
-        // Two groups of four warps (one per TMEM lane quadrant) take alternate chunks: group 0 (warps 2..5)
-        // the even ones, group 1 (warps 6..9) the odd ones.  Per chunk a group builds P~ = P (.) M, the scaled
-        // copies of Q and K, and later stores the chunk's outputs.
-        const int grp = (warp - TILE_W0) >> 2;
-        const int gt = tid - (TILE_W0 + 4 * grp) * 32;    // 0..127 inside the group
+        // All eight warps work on every chunk: P~ = P (.) M (the four warps of quadrants 0 and 1), the scaled
+        // copies of Q and K (everyone), and the outputs of the previous chunk (everyone: lanes = d_v).
+        const int tt = tid - TILE_W0 * 32;                // 0..255
         const int q = warp & 3;                           // TMEM lane quadrant
+        const int half = (warp - TILE_W0) >> 2;           // column half: 32 score columns / 32 output tokens
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
-        for (int c = grp; c < nc; c += 2) {
-            const int s = c & 1;                          // == grp: stage, P~ buffer, gate buffer and M buffer
+        uint8_t* ostg = tiles + OFF_OSTG;
+
+        // chunk c: TMEM -> bf16 [token][d_v] in the staging tile (two swizzled boxes) -> one TMA store;
+        // a ragged last chunk is copied out of the staging tile row by row instead
+        auto outputs = [&](int c) {
+            mbar_wait(&sh.o_full[0], c & 1, abortp, p.status);
+            tc_fence_after();
+            uint32_t r[32];
+            tmem_ld32(lane_addr + COL_O + 32 * half, r);
+            tc_wait_ld();
+            __syncwarp();
+            if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
+            if (warp == 4 && lane == 0) TL(2, c, 4);
+            const int valid = min(C, sq.len - tok0 - c * C);
+            if (c > 0) mbar_wait(&sh.stg_free, (c - 1) & 1, abortp, p.status);   // the previous store has read the tile
+            {
+                // element (token jj, d_v vc) of a swizzled box sits at jj*128 + (((vc>>3) ^ (jj&7)) << 4) + (vc&7)*2:
+                // eight base pointers (one per jj mod 8) leave one convert and one store per element
+                const int vc = (32 * q + lane) & 63;
+                uint8_t* base = ostg + (q >> 1) * 8192 + (32 * half) * 128 + (vc & 7) * 2;
+                uint8_t* pr[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) pr[x] = base + (((vc >> 3) ^ x) << 4);
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj)
+                    *reinterpret_cast<__nv_bfloat16*>(pr[jj & 7] + jj * 128) = __float2bfloat16_rn(__uint_as_float(r[jj]));
+            }
+            if (valid == C) fence_proxy_async_smem();
+            named_bar_sync(1, 256);
+            if (valid == C) {
+                if (tt == 0) {
+                    tma_store_3d(&map_o, ostg, 0, h, t0 + c * C);
+                    tma_store_3d(&map_o, ostg + 8192, 64, h, t0 + c * C);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                    mbar_arrive(&sh.stg_free);
+                }
+            } else {
+                // rows [0, valid): 16 pieces of 16 bytes per token row, read back from the swizzled boxes
+#pragma unroll 1
+                for (int idx = tt; idx < valid * 16; idx += 256) {
+                    const int row = idx >> 4, pc = idx & 15;             // piece pc covers d_v 8 pc .. 8 pc + 7
+                    const uint4 x = *reinterpret_cast<const uint4*>(ostg + (pc >> 3) * 8192 + row * 128 + (((pc & 7) ^ (row & 7)) << 4));
+                    *reinterpret_cast<uint4*>(og + ((size_t)(t0 + c * C + row) * p.H + h) * D + 8 * pc) = x;
+                }
+                named_bar_sync(1, 256);
+                if (tt == 0) mbar_arrive(&sh.stg_free);
+            }
+            if (warp == 4 && lane == 0) TL(2, c, 5);
+        };
+
+        // Iteration c builds the operands of chunk c (c < nc) and stores the outputs of chunk c-1 (c > 0); the
+        // outputs go first when they are already there, otherwise after the operands.  One code copy of each.
+        for (int c = 0; c <= nc; ++c) {
+            const int s = c & 1;
             GateSmem& gs = sh.gs[s];
             uint8_t* st = tiles + s * STAGE_BYTES;
-            const float* Mm = reinterpret_cast<const float*>(tiles + OFF_MASK + s * MASK_BYTES);
+            const uint8_t* Mm = tiles + OFF_MASK + s * MASK_BYTES;
             if (warp == 4 && lane == 0) TL(2, c, 0);
-            mbar_wait(&sh.m_ready[s], (c >> 1) & 1, abortp, p.status);
-            mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
-            mbar_wait(&sh.p_full[s], (c >> 1) & 1, abortp, p.status);   // P ready; the MMA is also done reading raw Q, K
-            tc_fence_after();
-            if (warp == 4 && lane == 0) TL(2, c, 1);
-            if (q < 2) {
-                // ---- P~ rows 32q..32q+31, all 64 columns
-                const int j = 32 * q + lane;
-                uint8_t* pt = tiles + OFF_PT + s * 8192;
-                uint32_t r0[32], r1[32];
-                tmem_ld32(lane_addr + COL_P, r0);
-                if (q == 1) tmem_ld32(lane_addr + COL_P + 32, r1);
-                tc_wait_ld();
-                __syncwarp();
-                if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
-                const float4* mrow = reinterpret_cast<const float4*>(Mm + j * MASK_PITCH);
-                auto half = [&](const uint32_t (&r)[32], int hcol) {   // 32 columns starting at hcol
+            bool out_done = c == 0;
+#pragma unroll 1
+            for (int pass = 0; pass < 2; ++pass) {
+                if (!out_done && (pass == 1 || c == nc || mbar_test_wait(&sh.o_full[0], (c - 1) & 1))) {
+                    outputs(c - 1);
+                    out_done = true;
+                }
+                if (pass == 1 || c == nc) continue;
+                mbar_wait(&sh.m_ready[s], (c >> 1) & 1, abortp, p.status);
+                mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
+                mbar_wait(&sh.p_full[0], c & 1, abortp, p.status);   // P ready; the MMA is also done reading raw Q, K
+                tc_fence_after();
+                if (warp == 4 && lane == 0) TL(2, c, 1);
+                if (q >= 2 && lane == 0) mbar_arrive(&sh.p_free);   // these warps do not read P; they only had to see this phase
+                if (q < 2) {
+                    // ---- P~ rows 32q..32q+31, columns 32 half .. +31
+                    const int j = 32 * q + lane;
+                    uint8_t* pt = tiles + OFF_PT + s * 8192;
+                    const bool any = half <= q;               // block not entirely above the diagonal
+                    uint32_t r[32];
+                    if (any) { tmem_ld32(lane_addr + COL_P + 32 * half, r); tc_wait_ld(); }
+                    __syncwarp();
+                    if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
+                    const uint4* mrow = reinterpret_cast<const uint4*>(Mm + j * (MASK_PITCH * 2) + 64 * half);
 #pragma unroll
                     for (int m4 = 0; m4 < 4; ++m4) {
                         uint32_t pk[4] = {0u, 0u, 0u, 0u};
-                        // columns hcol + 8 m4 .. +7 ; everything right of the row's 16-block is zero
-                        if (hcol + 8 * m4 <= (j | 15)) {
-                            const float4 ma = mrow[hcol / 4 + 2 * m4], mb = mrow[hcol / 4 + 2 * m4 + 1];
-                            const int o = 8 * m4;
-                            pk[0] = pack_bf16(__uint_as_float(r[o + 0]) * ma.x, __uint_as_float(r[o + 1]) * ma.y);
-                            pk[1] = pack_bf16(__uint_as_float(r[o + 2]) * ma.z, __uint_as_float(r[o + 3]) * ma.w);
-                            pk[2] = pack_bf16(__uint_as_float(r[o + 4]) * mb.x, __uint_as_float(r[o + 5]) * mb.y);
-                            pk[3] = pack_bf16(__uint_as_float(r[o + 6]) * mb.z, __uint_as_float(r[o + 7]) * mb.w);
+                        // columns 32 half + 8 m4 .. +7 ; everything right of the row's 16-block is zero
+                        if (any && 32 * half + 8 * m4 <= (j | 15)) {
+                            const uint4 mm = mrow[m4];
+                            const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162*>(&mw[e]);
+                                pk[e] = pack_bf16(__uint_as_float(r[8 * m4 + 2 * e]) * __low2float(m2),
+                                                  __uint_as_float(r[8 * m4 + 2 * e + 1]) * __high2float(m2));
+                            }
                         }
-                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, hcol + 8 * m4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 * half + 8 * m4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
-                };
-                half(r0, 0);
-                if (q == 1) {
-                    half(r1, 32);
-                } else {
-#pragma unroll
-                    for (int m4 = 0; m4 < 4; ++m4)
-                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 + 8 * m4)) = make_uint4(0u, 0u, 0u, 0u);
                 }
-            }
-            {
-                // ---- scaled copies: every thread of the group handles eight 16-byte pieces of Q and of K
-#pragma unroll 2
-                for (int m = 0; m < 8; ++m) {
-                    const int idx = gt + 128 * m;             // 16-byte piece inside a 16 KB tile
-                    const int row = (idx >> 3) & 63;
-                    uint4* qp = reinterpret_cast<uint4*>(st + OFF_Q) + idx;
-                    uint4* kp = reinterpret_cast<uint4*>(st + OFF_K) + idx;
-                    const uint4 xq = *qp, xk = *kp;
-                    const uint32_t f0 = gs.rowf[0][row], f1 = gs.rowf[1][row], w0 = gs.w[0][row], w1 = gs.w[1][row];
-                    *qp = scale8(xq, f0);
-                    *(qp + 1024) = scale8(xq, f1);
-                    *kp = scale8(xk, w0);
-                    *(kp + 1024) = scale8(xk, w1);
+                {
+                    // ---- scaled copies: every thread handles four 16-byte pieces of Q and of K
+#pragma unroll 1
+                    for (int m = 0; m < 4; ++m) {
+                        const int idx = tt + 256 * m;             // 16-byte piece inside a 16 KB tile
+                        const int row = (idx >> 3) & 63;
+                        uint4* qp = reinterpret_cast<uint4*>(st + OFF_Q) + idx;
+                        uint4* kp = reinterpret_cast<uint4*>(st + OFF_K) + idx;
+                        const uint4 xq = *qp, xk = *kp;
+                        const uint32_t f0 = gs.rowf[0][row], f1 = gs.rowf[1][row], w0 = gs.w[0][row], w1 = gs.w[1][row];
+                        *qp = scale8(xq, f0);
+                        *(qp + 1024) = scale8(xq, f1);
+                        *kp = scale8(xk, w0);
+                        *(kp + 1024) = scale8(xk, w1);
+                    }
                 }
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(&sh.prep_ready[s]); mbar_arrive(&sh.m_free[s]); }
-            if (warp == 4 && lane == 0) TL(2, c, 2);
-            // ---- outputs of this chunk: lanes = d_v, 64 token columns.  The readout is finished, so the stage's
-            // Q~ region is free: the tile is transposed into it as bf16 [token][d_v] (two swizzled boxes) and
-            // written out by one TMA store; a ragged last chunk is stored row by row instead.
-            mbar_wait(&sh.o_full[s], (c >> 1) & 1, abortp, p.status);
-            tc_fence_after();
-            if (warp == 4 && lane == 0) TL(2, c, 3);
-            const int valid = min(C, sq.len - tok0 - c * C);
-            {
-                uint32_t r0[32], r1[32];
-                tmem_ld32(lane_addr + COL_O, r0);
-                tmem_ld32(lane_addr + COL_O + 32, r1);
-                tc_wait_ld();
+                fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
-                if (warp == 4 && lane == 0) TL(2, c, 4);
-                if (valid == C) {
-                    uint8_t* box = st + OFF_Q + (q >> 1) * 8192;          // d_v half of this quadrant
-                    const int vc = (32 * q + lane) & 63;
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        *reinterpret_cast<__nv_bfloat16*>(box + sw128_offset(jj, vc)) = __float2bfloat16_rn(__uint_as_float(r0[jj]));
-                        *reinterpret_cast<__nv_bfloat16*>(box + sw128_offset(32 + jj, vc)) = __float2bfloat16_rn(__uint_as_float(r1[jj]));
-                    }
-                    fence_proxy_async_smem();
-                } else {
-                    __nv_bfloat16* orow = og + ((size_t)(t0 + c * C) * p.H + h) * D + 32 * q + lane;
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        if (jj < valid) orow[(size_t)jj * p.H * D] = __float2bfloat16_rn(__uint_as_float(r0[jj]));
-                        if (32 + jj < valid) orow[(size_t)(32 + jj) * p.H * D] = __float2bfloat16_rn(__uint_as_float(r1[jj]));
-                    }
-                }
+                if (lane == 0) { mbar_arrive(&sh.prep_ready[0]); mbar_arrive(&sh.m_free[s]); }
+                if (warp == 4 && lane == 0) TL(2, c, 2);
             }
-            named_bar_sync(3 + grp, 128);
-            if (gt == 0) {
-                if (valid == C) {
-                    tma_store_3d(&map_o, st + OFF_Q, 0, h, t0 + c * C);
-                    tma_store_3d(&map_o, st + OFF_Q + 8192, 64, h, t0 + c * C);
-                    tma_store_commit();
-                    tma_store_wait_read();       // the staging bytes have been read; the stage may be refilled
-                }
-                mbar_arrive(&sh.empty[s]);
-            }
-            if (warp == 4 && lane == 0) TL(2, c, 5);
         }
-        if (gt == 0) tma_store_wait_all();       // global writes of this group's stores are complete
+        if (tt == 0) tma_store_wait_all();       // global writes of the stores are complete
     } else if (warp >= GATE_W0) {
         // ------------------------------------------------------------------ gate warps 18,19
-        // Thread s owns token column s of the chunk.  One pass over the rows j multiplies gates together:
-        // d_i(j, s) = prod_{t = s+1..j} g^i_t (exact products: a zero gate gives an exact zero, no logs), so
-        //   M[j][s]   = W1 d_1 + W2 d_2                      (decay mask, 0 above the diagonal)
-        // and the per-token factors come from warp-wide prefix / suffix products:
-        //   w^i_s     = prod_{t > s} g^i_t                    (decay to the end of the chunk)
-        //   rowf^i_j  = W_i prod_{t <= j} g^i_t               (decay from the chunk start through token j)
-        const int sc = tid - GATE_W0 * 32;                // 0..63
+        // Running products of gates down the rows give the decay mask without logs or exps (a zero gate
+        // gives an exact zero): M[j][s] = W1 d_1(j,s) + W2 d_2(j,s), d_i(j,s) = prod_{t=s+1..j} g^i_t, 0 for s > j.
+        // Warp 18 owns columns 0..31 (rows 0..31 from 1, rows 32..63 continuing from the product to row 31),
+        // warp 19 columns 32..63 (rows 32..63).  The per-token factors come from warp-wide product scans:
+        //   w^i_s    = prod_{t > s} g^i_t                     (decay to the end of the chunk)
+        //   rowf^i_j = W_i prod_{t <= j} g^i_t                (decay from the chunk start through token j)
+        const int gw = warp - GATE_W0;
         const float gam = p.gamma[h];
         const float W1 = gam * p.scale, W2 = (1.f - gam) * p.scale;
         // each warp keeps all 64 gate pairs of the chunk in registers: lane l holds tokens l and l + 32
@@ -412,38 +494,53 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         for (int c = 0; c < nc; ++c) {
             const int s = c & 1;
             GateSmem& gs = sh.gs[s];
-            float* Mm = reinterpret_cast<float*>(tiles + OFF_MASK + s * MASK_BYTES);
+            __nv_bfloat16* Mm = reinterpret_cast<__nv_bfloat16*>(tiles + OFF_MASK + s * MASK_BYTES);
             const float2 glo = nlo, ghi = nhi;
             fetch(c + 1, nlo, nhi);
             if (c >= 2) mbar_wait(&sh.m_free[s], ((c >> 1) - 1) & 1, abortp, p.status);
             if (warp == GATE_W0 && lane == 0) TL(0, c, 1);
+            // suffix products of the lower half for both states (start values of rows 32..63 in columns 0..31)
+            const float slx = warp_suffix_prod(glo.x, lane), sly = warp_suffix_prod(glo.y, lane);
             {
-                // per-token factors by warp scans: warp 18 for the history state, warp 19 for the recency state
-                const int i = warp - GATE_W0;
-                const float xl = i == 0 ? glo.x : glo.y, xh = i == 0 ? ghi.x : ghi.y;   // tokens lane, lane + 32
-                const float Wi = i == 0 ? W1 : W2;
+                const float xl = gw == 0 ? glo.x : glo.y, xh = gw == 0 ? ghi.x : ghi.y;   // this warp's state
+                const float Wi = gw == 0 ? W1 : W2;
+                const float sl_in = gw == 0 ? slx : sly;
                 const float pl = warp_prefix_prod(xl, lane), ph0 = warp_prefix_prod(xh, lane);
                 const float tot_lo = __shfl_sync(0xffffffffu, pl, 31);
-                const float sh_in = warp_suffix_prod(xh, lane), sl_in = warp_suffix_prod(xl, lane);   // inclusive suffixes
+                const float sh_in = warp_suffix_prod(xh, lane);
                 const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0);
-                // exclusive suffix = inclusive suffix of the next lane (1 for the last token of each half)
                 float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
                 if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
                 const int valid = min(C, sq.len - tok0 - c * C);
-                gs.rowf[i][lane] = dup_bf16(Wi * pl);                       // decay from the chunk start through token j
-                gs.rowf[i][lane + 32] = dup_bf16(Wi * tot_lo * ph0);
+                gs.rowf[gw][lane] = dup_bf16(Wi * pl);
+                gs.rowf[gw][lane + 32] = dup_bf16(Wi * tot_lo * ph0);
                 // rows past the end of the sequence carry no weight in the state update
-                gs.w[i][lane] = dup_bf16(lane < valid ? sl_ex * tot_hi : 0.f);
-                gs.w[i][lane + 32] = dup_bf16(lane + 32 < valid ? sh_ex : 0.f);
+                gs.w[gw][lane] = dup_bf16(lane < valid ? sl_ex * tot_hi : 0.f);
+                gs.w[gw][lane + 32] = dup_bf16(lane + 32 < valid ? sh_ex : 0.f);
             }
-            float d1 = 1.f, d2 = 1.f;
-            float* mcol = Mm + sc;
-#pragma unroll 8
-            for (int j = 0; j < C; ++j) {
-                const float gx = __shfl_sync(0xffffffffu, j < 32 ? glo.x : ghi.x, j & 31);
-                const float gy = __shfl_sync(0xffffffffu, j < 32 ? glo.y : ghi.y, j & 31);
-                if (j > sc) { d1 *= gx; d2 *= gy; }
-                mcol[j * MASK_PITCH] = j >= sc ? fmaf(W2, d2, W1 * d1) : 0.f;
+            if (gw == 0) {
+                float ex = __shfl_down_sync(0xffffffffu, slx, 1), ey = __shfl_down_sync(0xffffffffu, sly, 1);
+                if (lane == 31) { ex = 1.f; ey = 1.f; }
+                float a1 = 1.f, a2 = 1.f, b1 = ex, b2 = ey;     // chains: rows 0..31 (triangle) and rows 32..63 (full)
+                __nv_bfloat16* mcol = Mm + lane;
+#pragma unroll 4
+                for (int jj = 0; jj < 32; ++jj) {
+                    const float gxa = __shfl_sync(0xffffffffu, glo.x, jj), gya = __shfl_sync(0xffffffffu, glo.y, jj);
+                    const float gxb = __shfl_sync(0xffffffffu, ghi.x, jj), gyb = __shfl_sync(0xffffffffu, ghi.y, jj);
+                    if (jj > lane) { a1 *= gxa; a2 *= gya; }
+                    b1 *= gxb; b2 *= gyb;
+                    mcol[jj * MASK_PITCH] = __float2bfloat16_rn(jj >= lane ? fmaf(W2, a2, W1 * a1) : 0.f);
+                    mcol[(32 + jj) * MASK_PITCH] = __float2bfloat16_rn(fmaf(W2, b2, W1 * b1));
+                }
+            } else {
+                float a1 = 1.f, a2 = 1.f;
+                __nv_bfloat16* mcol = Mm + 32 * MASK_PITCH + 32 + lane;
+#pragma unroll 4
+                for (int jj = 0; jj < 32; ++jj) {
+                    const float gx = __shfl_sync(0xffffffffu, ghi.x, jj), gy = __shfl_sync(0xffffffffu, ghi.y, jj);
+                    if (jj > lane) { a1 *= gx; a2 *= gy; }
+                    mcol[jj * MASK_PITCH] = __float2bfloat16_rn(jj >= lane ? fmaf(W2, a2, W1 * a1) : 0.f);
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.m_ready[s]);
@@ -474,40 +571,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             a_next = chunk_decay(c + 1);
             if (warp == 12 && lane == 0) TL(3, c, 0);
             if (c == 0) {
-                // initial state of this segment: slot contents (or zero) pushed through the summaries of
-                // the earlier segments, S <- A_j S + U_j; bf16 copy for the readout, a_0 S for the update
-                const float* base = slot1 + (size_t)hi * state_stride;
-                const float* wsu = tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr;
-#pragma unroll 1
-                for (int bt = 0; bt < 4; ++bt) {
-                    float acc[32];
-#pragma unroll
-                    for (int k = 0; k < 32; ++k)
-                        acc[k] = p.use_initial_state ? base[(size_t)(32 * bt + k) * D + v] : 0.f;
-                    for (int jg = 0; jg < g; ++jg) {
-                        const float* u = wsu + (size_t)jg * (SUMMARY_STRIDE / 4);
-                        const float A = u[2 * D * D + hi];
-                        const float* uu = u + (size_t)hi * D * D;
-#pragma unroll
-                        for (int k = 0; k < 32; ++k) acc[k] = fmaf(A, acc[k], uu[(size_t)(32 * bt + k) * D + v]);
-                    }
-                    uint32_t pk[16], sc[32];
-#pragma unroll
-                    for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(acc[2 * k], acc[2 * k + 1]);
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) sc[k] = __float_as_uint(acc[k] * a);
-                    tmem_st16(sb_addr + 16 * bt, pk);
-                    tmem_st32(s_addr + 32 * bt, sc);
-                }
+                init_state_pass(slot1 + (size_t)hi * state_stride, p.use_initial_state,
+                                tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, hi, v, a, s_addr, sb_addr);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(&sh.sb_ready); mbar_arrive(&sh.s_ready); }
+                if (lane == 0) { mbar_arrive(&sh.sb_ready[hi]); mbar_arrive(&sh.s_ready[hi]); }
                 continue;
             }
-            mbar_wait(&sh.u_full, (c - 1) & 1, abortp, p.status);
+            mbar_wait(&sh.u_full[hi], (c - 1) & 1, abortp, p.status);
             tc_fence_after();
             if (warp == 12 && lane == 0) TL(3, c, 1);
+            if (warp == 16 && lane == 0) TL(3, c, 4);
             // ---- A. bf16 copy of S_c: the readout of chunk c waits for this
             {
                 uint32_t r0[32], r1[32];
@@ -528,9 +603,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.sb_ready);
+                if (lane == 0) mbar_arrive(&sh.sb_ready[hi]);
             }
             if (warp == 12 && lane == 0) TL(3, c, 2);
+            if (warp == 16 && lane == 0) TL(3, c, 5);
             // ---- B. S <- a_c S: the state update of chunk c waits for this (it runs behind the readout MMAs)
             {
                 const float2 a2 = make_float2(a, a);
@@ -554,27 +630,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.s_ready);
+                if (lane == 0) mbar_arrive(&sh.s_ready[hi]);
             }
             if (warp == 12 && lane == 0) TL(3, c, 3);
+            if (warp == 16 && lane == 0) TL(3, c, 6);
         }
         // ---- final states of this segment's last chunk
-        mbar_wait(&sh.u_full, (nc - 1) & 1, abortp, p.status);
+        mbar_wait(&sh.u_full[hi], (nc - 1) & 1, abortp, p.status);
         tc_fence_after();
-        if (g == sq.last_seg) {
-            float* dst = slot1 + (size_t)hi * state_stride;
-#pragma unroll 1
-            for (int bt = 0; bt < 4; ++bt) {
-                uint32_t r[32];
-                tmem_ld32(s_addr + 32 * bt, r);
-                tc_wait_ld();
-#pragma unroll
-                for (int k = 0; k < 32; ++k) dst[(size_t)(32 * bt + k) * D + v] = __uint_as_float(r[k]);
-            }
-        }
+        if (g == sq.last_seg) store_state(slot1 + (size_t)hi * state_stride, v, s_addr);
     }
     tc_fence_before();
     __syncthreads();
+    if (tid == 0) TL(0, 63, 7);
     if (warp == WARP_MMA) tmem_dealloc(tb, 512);
 }
 
@@ -605,7 +673,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 
     if (tid == 0) {
         for (int s = 0; s < SUM_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        mbar_init(&sh.prep_ready[0], 8); mbar_init(&sh.u_full, 1);
+        mbar_init(&sh.prep_ready[0], 8); mbar_init(&sh.u_full[0], 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -645,7 +713,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) mma_ss(tb, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, (it | kk) > 0);
                 tc_commit(&sh.empty[s]);
-                if (it == nc - 1) tc_commit(&sh.u_full);
+                if (it == nc - 1) tc_commit(&sh.u_full[0]);
             }
         }
     } else {
@@ -696,7 +764,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             if (lane == 0) mbar_arrive(&sh.prep_ready[0]);
         }
         if (warp < 2 && lane == 0) out[2 * D * D + warp] = R;   // A_g: product of every gate of the segment
-        mbar_wait(&sh.u_full, 0, abortp, p.status);
+        mbar_wait(&sh.u_full[0], 0, abortp, p.status);
         tc_fence_after();
         {
             float* dst = out + (size_t)hi * D * D;
@@ -766,7 +834,8 @@ void plan(const dsla_prefill_args* a, int* nseg, int* cps) {
 }  // namespace
 
 #ifdef DSLA_TIMELINE
-extern "C" int dsla_debug_set_timeline(long long* dev_ptr) {
+extern "C" int dsla_debug_set_timeline(long long* dev_ptr, int block) {
+    cudaMemcpyToSymbol(g_timeline_block, &block, sizeof(block));
     return (int)cudaMemcpyToSymbol(g_timeline, &dev_ptr, sizeof(dev_ptr));
 }
 #endif

@@ -31,19 +31,36 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait.  Gives up after `limit` polls (each poll may itself suspend for a short,
+// Non-blocking test (try_wait may suspend the thread for a while before it reports "not yet").
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  The fast path (phase already complete) is a single inlined try_wait; otherwise a
+// non-inlined loop polls.  It gives up after `limit` polls (each poll may itself suspend for a short,
 // hardware-chosen time), raises *abort_flag (shared) and *status (global) and returns false.  Once the
 // abort flag is up every later wait returns at once, so a CTA that lost a signal still runs to
 // its end, frees its TMEM and exits instead of hanging.
-__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                      uint32_t limit = 4000000u) {
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    constexpr uint32_t limit = 8000000u;   // polls of some tens of nanoseconds each: a fraction of a second
     for (uint32_t i = 0; i < limit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_test_wait(bar, parity)) return true;
+        __nanosleep(20);   // a hot spin would take issue slots from the warps that are doing the work
         if ((i & 1023u) == 1023u && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(status, 5 /* DSLA_ERR_TIMEOUT */);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_test_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
