@@ -45,7 +45,7 @@ constexpr int SMEM_TILES = OFF_OSTG + 16384;
 constexpr int SMEM_DYN = SMEM_TILES + 1024;  // + alignment slack
 // summary kernel: 4 stages of [K/K~1][K~2][V]
 constexpr int SUM_STAGES = 4, SUM_STAGE_BYTES = 3 * 16384, SUM_OFF_V = 32768;
-constexpr int SUM_NTHREADS = 320, SUM_NCOMPUTE = 256;
+constexpr int SUM_NTHREADS = 384, SUM_NCOMPUTE = 256;
 constexpr int SUM_SMEM_DYN = SUM_STAGES * SUM_STAGE_BYTES + 1024;
 // TMEM columns
 constexpr uint32_t COL_S = 0;      // fp32 S1^T [0,128), S2^T [128,256)
@@ -58,6 +58,7 @@ constexpr size_t SUMMARY_STRIDE = 2 * D * D * sizeof(float) + 256;  // U (both s
 __device__ long long* g_timeline = nullptr;   // [role 4][chunk 64][event 8]
 __device__ int g_timeline_block = 0;
 #define TL(role, c, ev) do { if (tlp && (c) < 64) tlp[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr
 #else
 #define TL(role, c, ev) do { } while (0)
@@ -197,6 +198,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int tok0 = sq.c_begin * C;              // its index inside the sequence
     TL_INIT;
     if (tid == 0) TL(0, 63, 6);
+    if (tid == 0 && g_timeline) { g_timeline[2048 + 4 * blockIdx.x] = gtime(); unsigned sm; asm("mov.u32 %0, %smid;" : "=r"(sm)); g_timeline[2048 + 4 * blockIdx.x + 2] = sm; }
 
     if (tid == 0) {
         mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
@@ -643,6 +645,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (tid == 0) TL(0, 63, 7);
+    if (tid == 0 && g_timeline) g_timeline[2048 + 4 * blockIdx.x + 1] = gtime();
     if (warp == WARP_MMA) tmem_dealloc(tb, 512);
 }
 
@@ -651,12 +654,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 // The chunks are walked from the END of the segment backwards while a running product R^i of all
 // later gates is carried, so every token's weight prod_{t > s} g^i_t (to the end of the segment) is a
 // plain product: no logarithms, no rescaling of the accumulator, and a zero gate is exact.
-// Warps 0..7 scale K (warps 0 and 1 first derive the weights), warp 8 drives TMA, warp 9 issues MMAs.
+// A pure streaming pipeline, four chunks deep: warps 10, 11 derive the weights (one state each),
+// warps 0..7 scale K into the two weighted copies, warp 8 drives TMA, warp 9 issues the MMAs.
 // ============================================================================================
 __global__ void __launch_bounds__(SUM_NTHREADS, 1)
 prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const TcParams tp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
+    __shared__ alignas(16) uint32_t wts[SUM_STAGES][2][C];     // per-token weights, bf16 in both halves
+    __shared__ uint64_t w_ready[SUM_STAGES], w_free[SUM_STAGES], k_ready[SUM_STAGES];
     const PrefillParams& p = tp.p;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -672,8 +678,11 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     float* out = tp.ws + ((size_t)(n * p.H + h) * tp.nseg + g) * (SUMMARY_STRIDE / 4);
 
     if (tid == 0) {
-        for (int s = 0; s < SUM_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        mbar_init(&sh.prep_ready[0], 8); mbar_init(&sh.u_full[0], 1);
+        for (int s = 0; s < SUM_STAGES; ++s) {
+            mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1);
+            mbar_init(&w_ready[s], 2); mbar_init(&w_free[s], 8); mbar_init(&k_ready[s], 8);
+        }
+        mbar_init(&sh.u_full[0], 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -684,7 +693,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const uint32_t tb = sh.tmem_base;
     volatile int* abortp = &sh.abort_flag;
 
-    // iteration it = 0 .. nc-1 handles chunk nc-1-it
+    // iteration it = 0 .. nc-1 handles chunk nc-1-it; stage s = it % 4, use u = it / 4 of that stage
     if (warp == 8) {
         if (lane == 0) {
             prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
@@ -705,8 +714,8 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
             for (int it = 0; it < nc; ++it) {
-                const int s = it % SUM_STAGES;
-                mbar_wait(&sh.prep_ready[0], it & 1, abortp, p.status);
+                const int s = it % SUM_STAGES, u = it / SUM_STAGES;
+                mbar_wait(&k_ready[s], u & 1, abortp, p.status);
                 tc_fence_after();
                 const uint32_t st = sa + s * SUM_STAGE_BYTES;
                 const uint64_t dv = smem_desc_sw128(st + SUM_OFF_V, 8192, 1024), dkk = smem_desc_sw128(st, 8192, 1024);
@@ -716,68 +725,59 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                 if (it == nc - 1) tc_commit(&sh.u_full[0]);
             }
         }
+    } else if (warp >= 10) {
+        // ---- weights: warp 10 the history state, warp 11 the recency state; lane l holds tokens l and l + 32
+        const int i = warp - 10;
+        const float* gsrc = i == 0 ? p.g_hist : p.g_rec;
+        float R = 1.f;                                 // product of the gates of all later chunks
+        float nl = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + lane, p.H, h, true), 0.f);
+        float nh = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + lane + 32, p.H, h, true), 0.f);
+        for (int it = 0; it < nc; ++it) {
+            const int s = it % SUM_STAGES, u = it / SUM_STAGES;
+            const float xl = nl, xh = nh;
+            if (it + 1 < nc) {
+                const int t = t0 + (nc - 2 - it) * C + lane;
+                nl = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
+                nh = fmaxf(load_gate(gsrc, t + 32, p.H, h, true), 0.f);
+            }
+            const float sh_in = warp_suffix_prod(xh, lane), sl_in = warp_suffix_prod(xl, lane);
+            const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0), tot_lo = __shfl_sync(0xffffffffu, sl_in, 0);
+            float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
+            if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
+            if (u >= 1) mbar_wait(&w_free[s], (u - 1) & 1, abortp, p.status);
+            wts[s][i][lane] = dup_bf16(sl_ex * tot_hi * R);
+            wts[s][i][lane + 32] = dup_bf16(sh_ex * R);
+            R *= tot_lo * tot_hi;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&w_ready[s]);
+        }
+        if (lane == 0) out[2 * D * D + i] = R;         // A_g: product of every gate of the segment
     } else {
+        // ---- K~1 (in place) and K~2: four 16-byte pieces per thread and chunk
         const int q = warp & 3, hi = warp >> 2;
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
-        // warps 0 / 1: gates of the history / recency state, tokens lane and lane + 32 of the chunk
-        const float* gsrc = warp == 0 ? p.g_hist : p.g_rec;
-        float R = 1.f;                                 // product of the gates of all later chunks
-        float nl = 1.f, nh = 1.f;
-        if (warp < 2) {
-            const int t = t0 + (nc - 1) * C + lane;
-            nl = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
-            nh = fmaxf(load_gate(gsrc, t + 32, p.H, h, true), 0.f);
-        }
         for (int it = 0; it < nc; ++it) {
-            const int s = it % SUM_STAGES;
-            GateSmem& gs = sh.gs[it & 1];
+            const int s = it % SUM_STAGES, u = it / SUM_STAGES;
             uint8_t* st = tiles + s * SUM_STAGE_BYTES;
-            if (warp < 2) {
-                const float xl = nl, xh = nh;
-                if (it + 1 < nc) {
-                    const int t = t0 + (nc - 2 - it) * C + lane;
-                    nl = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
-                    nh = fmaxf(load_gate(gsrc, t + 32, p.H, h, true), 0.f);
-                }
-                const float sh_in = warp_suffix_prod(xh, lane), sl_in = warp_suffix_prod(xl, lane);
-                const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0), tot_lo = __shfl_sync(0xffffffffu, sl_in, 0);
-                float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
-                if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
-                gs.w[warp][lane] = dup_bf16(sl_ex * tot_hi * R);
-                gs.w[warp][lane + 32] = dup_bf16(sh_ex * R);
-                R *= tot_lo * tot_hi;
-            }
-            named_bar_sync(1, SUM_NCOMPUTE);
-            mbar_wait(&sh.full[s], (it / SUM_STAGES) & 1, abortp, p.status);
-#pragma unroll
+            mbar_wait(&w_ready[s], u & 1, abortp, p.status);
+            mbar_wait(&sh.full[s], u & 1, abortp, p.status);
+#pragma unroll 2
             for (int m = 0; m < 4; ++m) {
                 const int idx = tid + SUM_NCOMPUTE * m;
                 const int row = (idx >> 3) & 63;
                 uint4* kp = reinterpret_cast<uint4*>(st) + idx;
                 const uint4 xk = *kp;
-                const uint32_t w0 = gs.w[0][row], w1 = gs.w[1][row];
+                const uint32_t w0 = wts[s][0][row], w1 = wts[s][1][row];
                 *kp = scale8(xk, w0);
                 *(kp + 1024) = scale8(xk, w1);
             }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.prep_ready[0]);
+            if (lane == 0) { mbar_arrive(&k_ready[s]); mbar_arrive(&w_free[s]); }
         }
-        if (warp < 2 && lane == 0) out[2 * D * D + warp] = R;   // A_g: product of every gate of the segment
         mbar_wait(&sh.u_full[0], 0, abortp, p.status);
         tc_fence_after();
-        {
-            float* dst = out + (size_t)hi * D * D;
-            const int v = 32 * q + lane;
-#pragma unroll 1
-            for (int bt = 0; bt < 4; ++bt) {
-                uint32_t r[32];
-                tmem_ld32(lane_addr + 128 * hi + 32 * bt, r);
-                tc_wait_ld();
-#pragma unroll
-                for (int k = 0; k < 32; ++k) dst[(size_t)(32 * bt + k) * D + v] = __uint_as_float(r[k]);
-            }
-        }
+        store_state(out + (size_t)hi * D * D, 32 * q + lane, lane_addr + 128 * hi);
     }
     tc_fence_before();
     __syncthreads();
