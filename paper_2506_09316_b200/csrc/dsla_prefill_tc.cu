@@ -198,7 +198,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int tok0 = sq.c_begin * C;              // its index inside the sequence
     TL_INIT;
     if (tid == 0) TL(0, 63, 6);
-    if (tid == 0 && g_timeline) { g_timeline[2048 + 4 * blockIdx.x] = gtime(); unsigned sm; asm("mov.u32 %0, %smid;" : "=r"(sm)); g_timeline[2048 + 4 * blockIdx.x + 2] = sm; }
+#ifdef DSLA_TIMELINE
+    if (tid == 0 && g_timeline) g_timeline[2048 + 4 * blockIdx.x] = gtime();
+#endif
 
     if (tid == 0) {
         mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
@@ -645,7 +647,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (tid == 0) TL(0, 63, 7);
+#ifdef DSLA_TIMELINE
     if (tid == 0 && g_timeline) g_timeline[2048 + 4 * blockIdx.x + 1] = gtime();
+#endif
     if (warp == WARP_MMA) tmem_dealloc(tb, 512);
 }
 
