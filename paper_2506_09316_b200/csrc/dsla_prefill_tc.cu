@@ -59,8 +59,22 @@ __device__ long long* g_timeline = nullptr;   // [role 4][chunk 64][event 8]
 __device__ int g_timeline_block = 0;
 #define TL(role, c, ev) do { if (tlp && (c) < 64) tlp[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr
+#define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr; \
+    long long tl_w[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; const long long tl_t0 = clock64()
+// wait with the cycles it took added to this thread's counter `tag`; TL_DUMP writes a role's counters and its lifetime
+#define WAITP(tag, bar, ph) do { const long long _a = clock64(); mbar_wait(bar, ph, abortp, p.status); tl_w[tag] += clock64() - _a; } while (0)
+#define TLT(var) const long long var = clock64()
+#define TLACC(tag, expr) tl_w[tag] += (expr)
+#define TLW_BEGIN const long long _tlb = clock64()
+#define TLW_END(tag) tl_w[tag] += clock64() - _tlb
+#define TL_DUMP(role) do { if (tlp) { for (int _k = 0; _k < 10; ++_k) tlp[2700 + 12 * (role) + _k] = tl_w[_k]; tlp[2700 + 12 * (role) + 10] = clock64() - tl_t0; } } while (0)
 #else
+#define WAITP(tag, bar, ph) mbar_wait(bar, ph, abortp, p.status)
+#define TLT(var) do { } while (0)
+#define TLACC(tag, expr) do { } while (0)
+#define TLW_BEGIN do { } while (0)
+#define TLW_END(tag) do { } while (0)
+#define TL_DUMP(role) do { } while (0)
 #define TL(role, c, ev) do { } while (0)
 #define TL_INIT do { } while (0)
 #endif
@@ -204,7 +218,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
     if (tid == 0) {
         mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
-        mbar_init(&sh.empty[0], 1); mbar_init(&sh.empty[1], 1);
+        mbar_init(&sh.empty[0], 2); mbar_init(&sh.empty[1], 2);   // both issuers release a stage
         mbar_init(&sh.p_full[0], 1); mbar_init(&sh.p_free, 8);   // every tile warp passes p_full before P is overwritten
         mbar_init(&sh.prep_ready[0], 8);
         mbar_init(&sh.sb_ready[0], 4); mbar_init(&sh.sb_ready[1], 4); mbar_init(&sh.s_ready[0], 4); mbar_init(&sh.s_ready[1], 4);
@@ -223,13 +237,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     volatile int* abortp = &sh.abort_flag;
 
     if (warp == WARP_TMA) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer + state-update issuer
+        // This thread loads the tiles and also issues the state updates S^i^T += V^T K~i: they depend only on
+        // the state warps' rescale, so taking them off the other issuer's instruction stream lets the two
+        // MMA streams (outputs / state) go out in parallel.
         if (lane == 0) {
             prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-            for (int c = 0; c < nc; ++c) {
+            auto load_tile = [&](int c) {
                 const int s = c & 1;
-                if (c >= 2) mbar_wait(&sh.empty[s], ((c >> 1) & 1) ^ 1, abortp, p.status);
-                TL(0, c, 0);
                 uint8_t* st = tiles + s * STAGE_BYTES;
                 const int t = t0 + c * C;
                 mbar_arrive_expect_tx(&sh.full[s], 6 * 8192);
@@ -239,17 +254,44 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tma_load_3d(st + OFF_K + 8192, &map_k, &sh.full[s], 64, h, t);
                 tma_load_3d(st + OFF_V, &map_v, &sh.full[s], 0, h, t);
                 tma_load_3d(st + OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
-#ifdef DSLA_TIMELINE
-                mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
-                TL(0, c, 3);
-#endif
                 if (c + 2 < nc) {   // pull the tile after next into L2 while this one is in flight
                     const int t2 = t + 2 * C;
                     tma_prefetch_3d(&map_q, 0, h, t2); tma_prefetch_3d(&map_q, 64, h, t2);
                     tma_prefetch_3d(&map_k, 0, h, t2); tma_prefetch_3d(&map_k, 64, h, t2);
                     tma_prefetch_3d(&map_v, 0, h, t2); tma_prefetch_3d(&map_v, 64, h, t2);
                 }
+            };
+            load_tile(0);
+            if (nc > 1) load_tile(1);
+            const uint32_t sa = smem_u32(tiles);
+            constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
+            constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4);
+            const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
+#pragma unroll 1
+            for (int c = 0; c < nc; ++c) {
+                const int s = c & 1;
+                const uint64_t so = (uint64_t)s * STAGE_STEP;
+                WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
+#pragma unroll 1
+                for (int i = 0; i < 2; ++i) {
+                    WAITP(1, &sh.s_ready[i], c & 1);    // fp32 state i has been rescaled
+                    tc_fence_after();
+                    const uint64_t a = dv0 + so, b = dkn0 + so + (uint64_t)(i * (16384 >> 4));
+                    { TLW_BEGIN;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S + 128 * i, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
+                    tc_commit(&sh.u_full[i]);
+                    TLW_END(3); }
+                }
+                tc_commit(&sh.empty[s]);
+                TL(0, c, 5);
+                if (c + 2 < nc) {
+                    WAITP(2, &sh.empty[s], (c >> 1) & 1);   // both issuers' MMAs on this stage are done
+                    TL(0, c + 2, 0);
+                    { TLW_BEGIN; load_tile(c + 2); TLW_END(4); }
+                }
             }
+            TL_DUMP(0);
         }
     } else if (warp == WARP_MMA) {
         // ------------------------------------------------------------------ MMA issuer
@@ -258,11 +300,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OS = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OV = idesc_bf16(128, 64, 1, 0);
-            constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
             // Descriptors of stage 0; stage 1 and the k-steps are reached by adding constants to the address field.
             constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4), PT_STEP = (uint64_t)(8192 >> 4);
             const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dk0 = smem_desc_sw128(sa + OFF_K, 16, 1024);
-            const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
+            const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024);
             const uint64_t dp0 = smem_desc_sw128(sa + OFF_PT, 16, 1024);
             // One thread issues every MMA of the CTA.  Groups of four with compile-time operand steps cost about 45
             // cycles per issue (a rolled loop about 80), which keeps the issue rate above the tensor pipe's.
@@ -293,14 +334,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const uint64_t so = (uint64_t)s * STAGE_STEP;
                 // Scores of the next chunk go out as soon as its tile has landed and every tile warp has seen P_c:
                 // polled between the MMA groups of this chunk so the tile warps can start on the next one early.
-                // stage: 0 wait operands, 1 V part, 2/3 state parts, 4/5 state updates, 6 done
+                // stage: 0 V part (waits for the operands), 2/3 state parts, 6 done
                 bool p_next_done = c + 1 >= nc;
                 int stage = 0;
 #pragma unroll 1
                 for (uint32_t spin = 0; spin < 40000000u && !(p_next_done && stage == 6); ++spin) {
+#ifdef DSLA_TIMELINE
+                    const long long tl_a = clock64();
+                    const int tl_stage = stage; const bool tl_p = p_next_done;
+#endif
                     if (!p_next_done && mbar_test_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1) && mbar_test_wait(&sh.p_free, c & 1)) {
                         tc_fence_after();
-                        issue_p(c + 1);
+                        { TLW_BEGIN; issue_p(c + 1); TLW_END(4); }
                         p_next_done = true;
                         TL(1, c + 1, 7);
                     }
@@ -309,7 +354,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             TL(1, c, 1);
                             tc_fence_after();
                             // O^T = V^T P~^T + S1^T Q~1^T + S2^T Q~2^T ; the first part does not need the states
-                            run_ss4(tb + COL_O, dv0 + so, dp0 + (uint64_t)s * PT_STEP, S128{}, S2{}, ID_OV, 0);
+                            { TLW_BEGIN; run_ss4(tb + COL_O, dv0 + so, dp0 + (uint64_t)s * PT_STEP, S128{}, S2{}, ID_OV, 0); TLW_END(2); }
                             stage = 2;
                         }
                     } else if (stage == 2 || stage == 3) {
@@ -319,27 +364,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             if (i == 0) TL(1, c, 3);
                             tc_fence_after();
                             const uint64_t dq = dq0 + so + (uint64_t)(i * (16384 >> 4));
+                            { TLW_BEGIN;
                             run_ts4(tb + COL_O, tb + COL_SB + 64 * i, dq, ID_OS);
                             run_ts4(tb + COL_O, tb + COL_SB + 64 * i + 32, dq + 512, ID_OS);
-                            if (i == 1) { tc_commit(&sh.o_full[0]); TL(1, c, 6); }
-                            ++stage;
-                        }
-                    } else if (stage == 4 || stage == 5) {
-                        // S^i^T += V^T K~i   (needs the rescaled fp32 state i)
-                        const int i = stage - 4;
-                        if (mbar_test_wait(&sh.s_ready[i], c & 1)) {
-                            if (i == 0) TL(1, c, 4);
-                            tc_fence_after();
-                            run_ss4(tb + COL_S + 128 * i, dv0 + so, dkn0 + so + (uint64_t)(i * (16384 >> 4)), S128{}, S128{}, ID_U, 1);
-                            tc_commit(&sh.u_full[i]);
-                            if (i == 1) { tc_commit(&sh.empty[s]); TL(1, c, 5); }
-                            ++stage;
+                            TLW_END(3); }
+                            if (i == 1) { TLW_BEGIN; tc_commit(&sh.o_full[0]); tc_commit(&sh.empty[s]); TLW_END(5); TL(1, c, 6); }
+                            stage = i == 0 ? 3 : 6;
                         }
                     }
+#ifdef DSLA_TIMELINE
+                    if (tl_stage != stage || tl_p != p_next_done) TLACC(1, clock64() - tl_a); else TLACC(0, clock64() - tl_a);
+#endif
                     if ((spin & 4095u) == 4095u && *abortp) break;
                 }
                 if (!(p_next_done && stage == 6) && !*abortp) { *abortp = 1; atomicExch(p.status, 5); }
             }
+            TL_DUMP(1);
         }
     } else if (warp < STATE_W0) {
         // ------------------------------------------------------------------ tile warps 2..9
@@ -355,16 +395,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // chunk c: TMEM -> bf16 [token][d_v] in the staging tile (two swizzled boxes) -> one TMA store;
         // a ragged last chunk is copied out of the staging tile row by row instead
         auto outputs = [&](int c) {
-            mbar_wait(&sh.o_full[0], c & 1, abortp, p.status);
+            WAITP(0, &sh.o_full[0], c & 1);
             tc_fence_after();
+            TLT(tlo0);
             uint32_t r[32];
             tmem_ld32(lane_addr + COL_O + 32 * half, r);
             tc_wait_ld();
+            TLT(tlo1); TLACC(5, tlo1 - tlo0);
             __syncwarp();
             if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
             if (warp == 4 && lane == 0) TL(2, c, 4);
             const int valid = min(C, sq.len - tok0 - c * C);
-            if (c > 0) mbar_wait(&sh.stg_free, (c - 1) & 1, abortp, p.status);   // the previous store has read the tile
+            if (c > 0) WAITP(1, &sh.stg_free, (c - 1) & 1);   // the previous store has read the tile
             {
                 // element (token jj, d_v vc) of a swizzled box sits at jj*128 + (((vc>>3) ^ (jj&7)) << 4) + (vc&7)*2:
                 // eight base pointers (one per jj mod 8) leave one convert and one store per element
@@ -377,6 +419,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 for (int jj = 0; jj < 32; ++jj)
                     *reinterpret_cast<__nv_bfloat16*>(pr[jj & 7] + jj * 128) = __float2bfloat16_rn(__uint_as_float(r[jj]));
             }
+            TLT(tlo2); TLACC(6, tlo2 - tlo1);
             if (valid == C) fence_proxy_async_smem();
             named_bar_sync(1, 256);
             if (valid == C) {
@@ -398,6 +441,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 named_bar_sync(1, 256);
                 if (tt == 0) mbar_arrive(&sh.stg_free);
             }
+            TLACC(7, clock64() - tlo2);
             if (warp == 4 && lane == 0) TL(2, c, 5);
         };
 
@@ -417,11 +461,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     out_done = true;
                 }
                 if (pass == 1 || c == nc) continue;
-                mbar_wait(&sh.m_ready[s], (c >> 1) & 1, abortp, p.status);
-                mbar_wait(&sh.full[s], (c >> 1) & 1, abortp, p.status);
-                mbar_wait(&sh.p_full[0], c & 1, abortp, p.status);   // P ready; the MMA is also done reading raw Q, K
+                WAITP(2, &sh.m_ready[s], (c >> 1) & 1);
+                WAITP(3, &sh.full[s], (c >> 1) & 1);
+                WAITP(4, &sh.p_full[0], c & 1);   // P ready; the MMA is also done reading raw Q, K
                 tc_fence_after();
                 if (warp == 4 && lane == 0) TL(2, c, 1);
+                TLT(tlm0);
                 if (q >= 2 && lane == 0) mbar_arrive(&sh.p_free);   // these warps do not read P; they only had to see this phase
                 if (q < 2) {
                     // ---- P~ rows 32q..32q+31, columns 32 half .. +31
@@ -450,6 +495,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 * half + 8 * m4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 }
+                TLT(tlm1); TLACC(8, tlm1 - tlm0);
                 {
                     // ---- scaled copies: every thread handles four 16-byte pieces of Q and of K
 #pragma unroll 1
@@ -466,12 +512,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         *(kp + 1024) = scale8(xk, w1);
                     }
                 }
+                TLACC(9, clock64() - tlm1);
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.prep_ready[0]); mbar_arrive(&sh.m_free[s]); }
                 if (warp == 4 && lane == 0) TL(2, c, 2);
             }
         }
+        if (warp == 4 && lane == 0) TL_DUMP(2);
+        if (warp == 6 && lane == 0) TL_DUMP(3);
         if (tt == 0) tma_store_wait_all();       // global writes of the stores are complete
     } else if (warp >= GATE_W0) {
         // ------------------------------------------------------------------ gate warps 18,19
@@ -501,8 +550,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             __nv_bfloat16* Mm = reinterpret_cast<__nv_bfloat16*>(tiles + OFF_MASK + s * MASK_BYTES);
             const float2 glo = nlo, ghi = nhi;
             fetch(c + 1, nlo, nhi);
-            if (c >= 2) mbar_wait(&sh.m_free[s], ((c >> 1) - 1) & 1, abortp, p.status);
+            if (c >= 2) WAITP(0, &sh.m_free[s], ((c >> 1) - 1) & 1);
             if (warp == GATE_W0 && lane == 0) TL(0, c, 1);
+            TLT(tlg0);
             // suffix products of the lower half for both states (start values of rows 32..63 in columns 0..31)
             const float slx = warp_suffix_prod(glo.x, lane), sly = warp_suffix_prod(glo.y, lane);
             {
@@ -522,6 +572,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 gs.w[gw][lane] = dup_bf16(lane < valid ? sl_ex * tot_hi : 0.f);
                 gs.w[gw][lane + 32] = dup_bf16(lane + 32 < valid ? sh_ex : 0.f);
             }
+            TLT(tlg1); TLACC(1, tlg1 - tlg0);
             if (gw == 0) {
                 float ex = __shfl_down_sync(0xffffffffu, slx, 1), ey = __shfl_down_sync(0xffffffffu, sly, 1);
                 if (lane == 31) { ex = 1.f; ey = 1.f; }
@@ -546,10 +597,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     mcol[jj * MASK_PITCH] = __float2bfloat16_rn(jj >= lane ? fmaf(W2, a2, W1 * a1) : 0.f);
                 }
             }
+            TLACC(2, clock64() - tlg1);
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.m_ready[s]);
             if (warp == GATE_W0 && lane == 0) TL(0, c, 2);
         }
+        if (warp == GATE_W0 && lane == 0) TL_DUMP(6);
     } else {
         // ------------------------------------------------------------------ state warps 10..17
         const int q = warp & 3, hi = (warp - STATE_W0) >> 2;   // TMEM lane quadrant, state index
@@ -558,21 +611,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const uint32_t sb_addr = lane_addr + COL_SB + 64 * hi;
         const int v = 32 * q + lane;
         const float* gsrc = hi == 0 ? p.g_hist : p.g_rec;
-        // chunk decay a = prod of this state's gates over the chunk (two tokens per lane), fetched one chunk ahead
-        auto chunk_decay = [&](int c) -> float {
+        // chunk decay a = prod of this state's gates over the chunk (two tokens per lane).  The gates of chunk c + 1
+        // are requested at the top of iteration c and multiplied together at its end, so the load latency hides
+        // behind the waits and the two passes.
+        auto gate_pair = [&](int c) -> float2 {
             const int j = c * C + 2 * lane;
             const bool in = c < nc;
-            const float ga = load_gate(gsrc, t0 + j, p.H, h, in && tok0 + j < sq.len);
-            const float gb = load_gate(gsrc, t0 + j + 1, p.H, h, in && tok0 + j + 1 < sq.len);
-            float pr = fmaxf(ga, 0.f) * fmaxf(gb, 0.f);
+            return make_float2(load_gate(gsrc, t0 + j, p.H, h, in && tok0 + j < sq.len),
+                               load_gate(gsrc, t0 + j + 1, p.H, h, in && tok0 + j + 1 < sq.len));
+        };
+        auto warp_prod = [&](float2 gp) -> float {
+            float pr = fmaxf(gp.x, 0.f) * fmaxf(gp.y, 0.f);
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) pr *= __shfl_xor_sync(0xffffffffu, pr, off);
             return pr;
         };
-        float a_next = chunk_decay(0);
+        float a_next = warp_prod(gate_pair(0));
         for (int c = 0; c < nc; ++c) {
             const float a = a_next;
-            a_next = chunk_decay(c + 1);
+            const float2 gp_next = gate_pair(c + 1);
             if (warp == 12 && lane == 0) TL(3, c, 0);
             if (c == 0) {
                 init_state_pass(slot1 + (size_t)hi * state_stride, p.use_initial_state,
@@ -581,12 +638,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.sb_ready[hi]); mbar_arrive(&sh.s_ready[hi]); }
+                a_next = warp_prod(gp_next);
                 continue;
             }
-            mbar_wait(&sh.u_full[hi], (c - 1) & 1, abortp, p.status);
+            WAITP(0, &sh.u_full[hi], (c - 1) & 1);
+            WAITP(1, &sh.o_full[0], (c - 1) & 1);   // the readout of chunk c-1 (other issuer) has read the bf16 copy
             tc_fence_after();
             if (warp == 12 && lane == 0) TL(3, c, 1);
             if (warp == 16 && lane == 0) TL(3, c, 4);
+            TLT(tls0);
             // ---- A. bf16 copy of S_c: the readout of chunk c waits for this
             {
                 uint32_t r0[32], r1[32];
@@ -611,6 +671,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
             if (warp == 12 && lane == 0) TL(3, c, 2);
             if (warp == 16 && lane == 0) TL(3, c, 5);
+            TLT(tls1); TLACC(2, tls1 - tls0);
             // ---- B. S <- a_c S: the state update of chunk c waits for this (it runs behind the readout MMAs)
             {
                 const float2 a2 = make_float2(a, a);
@@ -636,9 +697,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.s_ready[hi]);
             }
+            TLACC(3, clock64() - tls1);
+            a_next = warp_prod(gp_next);
             if (warp == 12 && lane == 0) TL(3, c, 3);
             if (warp == 16 && lane == 0) TL(3, c, 6);
         }
+        if (warp == 12 && lane == 0) TL_DUMP(4);
+        if (warp == 16 && lane == 0) TL_DUMP(5);
         // ---- final states of this segment's last chunk
         mbar_wait(&sh.u_full[hi], (nc - 1) & 1, abortp, p.status);
         tc_fence_after();
