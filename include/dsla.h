@@ -115,8 +115,10 @@ typedef struct {
     size_t workspace_bytes;
 } dsla_prefill_args;
 
-/* Scratch the chosen kernel needs for these sizes (0 for the SIMT kernel).  Pointers in `a` are
- * not dereferenced. */
+/* Scratch the chosen kernel needs for these sizes (0 for the SIMT kernel): the segment summaries of
+ * sequences that are split along T, plus, for packed batches (cu_seqlens != NULL, N > 1), one int32 per
+ * sequence for the longest-first visiting order.  Pointers in `a` are not dereferenced (cu_seqlens is
+ * only compared with NULL). */
 size_t dsla_prefill_workspace_bytes(const dsla_prefill_args* a);
 
 /* Writes o for every token and the final states of every sequence into its slot.  A sequence of

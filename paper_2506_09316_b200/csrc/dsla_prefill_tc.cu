@@ -40,8 +40,7 @@ constexpr int OFF_PT = 2 * STAGE_BYTES;  // P~ double buffer, 8 KB each
 constexpr int OFF_MASK = OFF_PT + 2 * 8192;  // decay mask M, bf16 [2][64][MASK_PITCH] (one buffer per chunk parity)
 constexpr int MASK_PITCH = 72;               // bf16 elements; 144-byte rows keep 16-byte row accesses conflict-free
 constexpr int MASK_BYTES = 64 * MASK_PITCH * 2;
-constexpr int OFF_OSTG = OFF_MASK + 2 * MASK_BYTES + 1024 - (2 * MASK_BYTES) % 1024;   // output staging, 2 x 8 KB boxes
-constexpr int SMEM_TILES = OFF_OSTG + 16384;
+constexpr int SMEM_TILES = OFF_MASK + 2 * MASK_BYTES;
 constexpr int SMEM_DYN = SMEM_TILES + 1024;  // + alignment slack
 // summary kernel: 4 stages of [K/K~1][K~2][V]
 constexpr int SUM_STAGES = 4, SUM_STAGE_BYTES = 3 * 16384, SUM_OFF_V = 32768;
@@ -57,7 +56,7 @@ constexpr size_t SUMMARY_STRIDE = 2 * D * D * sizeof(float) + 256;  // U (both s
 #ifdef DSLA_TIMELINE
 __device__ long long* g_timeline = nullptr;   // [role 4][chunk 64][event 8]
 __device__ int g_timeline_block = 0;
-#define TL(role, c, ev) do { if (tlp && (c) < 64) tlp[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
+#define TL(role, c, ev) do { if (tlp && (unsigned)(c) < 64u) tlp[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr; \
     long long tl_w[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; const long long tl_t0 = clock64()
@@ -84,6 +83,7 @@ struct TcParams {
     float* ws;          // summaries: [(n*H + h)*nseg + g] -> {U[2][D][D], A[2]}
     int nseg;           // segments per sequence (grid dimension)
     int cps;            // chunks per segment
+    const int* order;   // sequences by descending length (longest first), or nullptr for index order
 };
 
 // Per-token factors of one chunk, per state.
@@ -93,7 +93,7 @@ struct alignas(16) GateSmem {
 };
 
 struct alignas(16) Shared {
-    uint64_t full[4], empty[4], p_full[2], p_free, prep_ready[2], sb_ready[2], s_ready[2], o_full[2], o_free, u_full[2], m_ready[2], m_free[2], stg_free;
+    uint64_t full[4], empty[4], p_full[2], p_free, prep_ready[2], sb_ready[2], s_ready[2], o_full[2], o_free, u_full[2], m_ready[2], m_free[2];
     uint32_t tmem_base;
     int abort_flag;
     GateSmem gs[2];
@@ -188,7 +188,7 @@ __device__ __noinline__ void store_state(float* dst, int v, uint32_t s_addr) {
 // ============================================================================================
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, const TcParams tp) {
+                  const __grid_constant__ CUtensorMap map_v, const TcParams tp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ Shared sh;
     const PrefillParams& p = tp.p;
@@ -196,7 +196,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x % tp.nseg;
     const int h = (blockIdx.x / tp.nseg) % p.H;
-    const int n = blockIdx.x / (tp.nseg * p.H);
+    const int rank = blockIdx.x / (tp.nseg * p.H);
+    const int n = tp.order ? tp.order[rank] : rank;
     const SeqInfo sq = seq_info(p, n, g, tp.cps);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
     float* slot1 = p.state + (((size_t)sq.slot * 2) * p.H + h) * (size_t)(D * D);
@@ -225,7 +226,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(&sh.o_full[0], 1); mbar_init(&sh.o_free, 8); mbar_init(&sh.u_full[0], 1); mbar_init(&sh.u_full[1], 1);
         mbar_init(&sh.m_ready[0], 2); mbar_init(&sh.m_ready[1], 2);
         mbar_init(&sh.m_free[0], 8); mbar_init(&sh.m_free[1], 8);
-        mbar_init(&sh.stg_free, 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -261,19 +261,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     tma_prefetch_3d(&map_v, 0, h, t2); tma_prefetch_3d(&map_v, 64, h, t2);
                 }
             };
-            load_tile(0);
-            if (nc > 1) load_tile(1);
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
             constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4);
             const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
+            // iterations -2 and -1 only start the first two loads (one copy of the load code)
 #pragma unroll 1
-            for (int c = 0; c < nc; ++c) {
+            for (int c = -2; c < nc; ++c) {
                 const int s = c & 1;
                 const uint64_t so = (uint64_t)s * STAGE_STEP;
-                WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
+                if (c >= 0) WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
 #pragma unroll 1
-                for (int i = 0; i < 2; ++i) {
+                for (int i = 0; i < 2 && c >= 0; ++i) {
                     WAITP(1, &sh.s_ready[i], c & 1);    // fp32 state i has been rescaled
                     tc_fence_after();
                     const uint64_t a = dv0 + so, b = dkn0 + so + (uint64_t)(i * (16384 >> 4));
@@ -283,10 +282,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     tc_commit(&sh.u_full[i]);
                     TLW_END(3); }
                 }
-                tc_commit(&sh.empty[s]);
+                if (c >= 0) tc_commit(&sh.empty[s]);
                 TL(0, c, 5);
                 if (c + 2 < nc) {
-                    WAITP(2, &sh.empty[s], (c >> 1) & 1);   // both issuers' MMAs on this stage are done
+                    if (c >= 0) WAITP(2, &sh.empty[s], (c >> 1) & 1);   // both issuers' MMAs on this stage are done
                     TL(0, c + 2, 0);
                     { TLW_BEGIN; load_tile(c + 2); TLW_END(4); }
                 }
@@ -390,10 +389,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int half = (warp - TILE_W0) >> 2;           // column half: 32 score columns / 32 output tokens
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
-        uint8_t* ostg = tiles + OFF_OSTG;
 
-        // chunk c: TMEM -> bf16 [token][d_v] in the staging tile (two swizzled boxes) -> one TMA store;
-        // a ragged last chunk is copied out of the staging tile row by row instead
+        // chunk c: each thread owns one d_v lane of O^T and 32 tokens; a warp's store of one token is 64 contiguous
+        // bytes (two full sectors), so the outputs go straight from registers to global memory
         auto outputs = [&](int c) {
             WAITP(0, &sh.o_full[0], c & 1);
             tc_fence_after();
@@ -405,43 +403,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             __syncwarp();
             if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
             if (warp == 4 && lane == 0) TL(2, c, 4);
-            const int valid = min(C, sq.len - tok0 - c * C);
-            if (c > 0) WAITP(1, &sh.stg_free, (c - 1) & 1);   // the previous store has read the tile
-            {
-                // element (token jj, d_v vc) of a swizzled box sits at jj*128 + (((vc>>3) ^ (jj&7)) << 4) + (vc&7)*2:
-                // eight base pointers (one per jj mod 8) leave one convert and one store per element
-                const int vc = (32 * q + lane) & 63;
-                uint8_t* base = ostg + (q >> 1) * 8192 + (32 * half) * 128 + (vc & 7) * 2;
-                uint8_t* pr[8];
+            const int valid = min(C, sq.len - tok0 - c * C) - 32 * half;     // tokens of this warp's half that exist
+            __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * half) * p.H + h) * D + 32 * q + lane;
+            const size_t row = (size_t)p.H * D;
+            if (valid >= 32) {
 #pragma unroll
-                for (int x = 0; x < 8; ++x) pr[x] = base + (((vc >> 3) ^ x) << 4);
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj)
-                    *reinterpret_cast<__nv_bfloat16*>(pr[jj & 7] + jj * 128) = __float2bfloat16_rn(__uint_as_float(r[jj]));
-            }
-            TLT(tlo2); TLACC(6, tlo2 - tlo1);
-            if (valid == C) fence_proxy_async_smem();
-            named_bar_sync(1, 256);
-            if (valid == C) {
-                if (tt == 0) {
-                    tma_store_3d(&map_o, ostg, 0, h, t0 + c * C);
-                    tma_store_3d(&map_o, ostg + 8192, 64, h, t0 + c * C);
-                    tma_store_commit();
-                    tma_store_wait_read();
-                    mbar_arrive(&sh.stg_free);
-                }
+                for (int jj = 0; jj < 32; ++jj) dst[jj * row] = __float2bfloat16_rn(__uint_as_float(r[jj]));
             } else {
-                // rows [0, valid): 16 pieces of 16 bytes per token row, read back from the swizzled boxes
 #pragma unroll 1
-                for (int idx = tt; idx < valid * 16; idx += 256) {
-                    const int row = idx >> 4, pc = idx & 15;             // piece pc covers d_v 8 pc .. 8 pc + 7
-                    const uint4 x = *reinterpret_cast<const uint4*>(ostg + (pc >> 3) * 8192 + row * 128 + (((pc & 7) ^ (row & 7)) << 4));
-                    *reinterpret_cast<uint4*>(og + ((size_t)(t0 + c * C + row) * p.H + h) * D + 8 * pc) = x;
+                for (int jj = 0; jj < valid; ++jj) {   // ragged tail (cold): pick the register with a shuffle-free select chain
+                    float x = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x = e == jj ? __uint_as_float(r[e]) : x;
+                    dst[jj * row] = __float2bfloat16_rn(x);
                 }
-                named_bar_sync(1, 256);
-                if (tt == 0) mbar_arrive(&sh.stg_free);
             }
-            TLACC(7, clock64() - tlo2);
+            TLACC(6, clock64() - tlo1);
             if (warp == 4 && lane == 0) TL(2, c, 5);
         };
 
@@ -521,7 +498,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         if (warp == 4 && lane == 0) TL_DUMP(2);
         if (warp == 6 && lane == 0) TL_DUMP(3);
-        if (tt == 0) tma_store_wait_all();       // global writes of the stores are complete
     } else if (warp >= GATE_W0) {
         // ------------------------------------------------------------------ gate warps 18,19
         // Running products of gates down the rows give the decay mask without logs or exps (a zero gate
@@ -738,7 +714,8 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const int nsum = tp.nseg - 1;
     const int g = blockIdx.x % nsum;
     const int h = (blockIdx.x / nsum) % p.H;
-    const int n = blockIdx.x / (nsum * p.H);
+    const int rank = blockIdx.x / (nsum * p.H);
+    const int n = tp.order ? tp.order[rank] : rank;
     const SeqInfo sq = seq_info(p, n, g, tp.cps);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
     if (sq.len <= 0 || g >= sq.last_seg) return;      // only segments that have a successor
@@ -888,6 +865,27 @@ bool make_map(CUtensorMap* m, const void* base, int T_total, int H) {
 
 // Segments per sequence: enough CTAs to cover the SMs when there are few (sequence, head) pairs,
 // never shorter than 4 chunks per segment.
+// Ragged batches: blocks are handed to the SMs in index order, so sequences are visited longest first (a long
+// sequence that starts late would otherwise run on alone at the end).  order[r] = index of the r-th longest
+// sequence, ties by index; one thread per sequence counts how many sequences come before its own.
+constexpr int ORDER_MAX_N = 8192;
+__global__ void seq_order_kernel(const int32_t* __restrict__ cu, int N, int* __restrict__ order) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    const int len_i = cu[i + 1] - cu[i];
+    int before = 0;
+    int prev = __ldg(cu);
+    for (int j = 0; j < N; ++j) {
+        const int next = __ldg(cu + j + 1);
+        const int len_j = next - prev;
+        prev = next;
+        before += (len_j > len_i || (len_j == len_i && j < i)) ? 1 : 0;
+    }
+    order[before] = i;
+}
+
+bool wants_order(const dsla_prefill_args* a) { return a->cu_seqlens != nullptr && a->N > 1 && a->N <= ORDER_MAX_N; }
+
 void plan(const dsla_prefill_args* a, int* nseg, int* cps) {
     const int max_chunks = (a->max_seqlen + C - 1) / C;
     const long long units = (long long)a->N * a->H;
@@ -914,8 +912,9 @@ bool prefill_tc_available() { return true; }
 size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a) {
     int nseg, cps;
     plan(a, &nseg, &cps);
-    if (nseg <= 1) return 0;
-    return (size_t)a->N * a->H * nseg * SUMMARY_STRIDE;
+    const size_t summaries = nseg > 1 ? (size_t)a->N * a->H * nseg * SUMMARY_STRIDE : 0;     // a multiple of 256
+    const size_t order = wants_order(a) ? (((size_t)a->N * sizeof(int) + 255) & ~(size_t)255) : 0;
+    return summaries + order;
 }
 
 dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a, cudaStream_t s) {
@@ -927,9 +926,16 @@ dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a
     tp.p = p;
     plan(a, &tp.nseg, &tp.cps);
     tp.ws = tp.nseg > 1 ? static_cast<float*>(a->workspace) : nullptr;
-    CUtensorMap mq, mk, mv, mo;
-    if (!make_map(&mq, p.q, a->T_total, p.H) || !make_map(&mk, p.k, a->T_total, p.H) || !make_map(&mv, p.v, a->T_total, p.H) ||
-        !make_map(&mo, p.o, a->T_total, p.H))
+    tp.order = nullptr;
+    if (wants_order(a)) {
+        const size_t summaries = tp.nseg > 1 ? (size_t)a->N * a->H * tp.nseg * SUMMARY_STRIDE : 0;
+        int* order = reinterpret_cast<int*>(static_cast<char*>(a->workspace) + summaries);
+        seq_order_kernel<<<dim3((unsigned)((p.N + 255) / 256)), dim3(256), 0, s>>>(p.cu_seqlens, p.N, order);
+        count_launch();
+        tp.order = order;
+    }
+    CUtensorMap mq, mk, mv;
+    if (!make_map(&mq, p.q, a->T_total, p.H) || !make_map(&mk, p.k, a->T_total, p.H) || !make_map(&mv, p.v, a->T_total, p.H))
         return DSLA_ERR_CUDA;
     if (cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN) != cudaSuccess ||
         cudaFuncSetAttribute(prefill_tc_summary_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SUM_SMEM_DYN) != cudaSuccess)
@@ -940,7 +946,7 @@ dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a
         prefill_tc_summary_kernel<<<dim3((unsigned)(units * (tp.nseg - 1))), dim3(SUM_NTHREADS), SUM_SMEM_DYN, s>>>(mk, mv, tp);
         count_launch();
     }
-    prefill_tc_kernel<<<dim3((unsigned)(units * tp.nseg)), dim3(NTHREADS), SMEM_DYN, s>>>(mq, mk, mv, mo, tp);
+    prefill_tc_kernel<<<dim3((unsigned)(units * tp.nseg)), dim3(NTHREADS), SMEM_DYN, s>>>(mq, mk, mv, tp);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
 }
