@@ -237,146 +237,120 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     volatile int* abortp = &sh.abort_flag;
 
     if (warp == WARP_TMA) {
-        // ------------------------------------------------------------------ TMA producer + state-update issuer
-        // This thread loads the tiles and also issues the state updates S^i^T += V^T K~i: they depend only on
-        // the state warps' rescale, so taking them off the other issuer's instruction stream lets the two
-        // MMA streams (outputs / state) go out in parallel.
+        // ------------------------------------------------------------------ TMA producer + issuer of P and the state updates
+        // Two threads issue the MMAs of a chunk.  This one loads the tiles, issues the scores P = Q K^T of the next
+        // chunk as soon as its tile has landed and P of this chunk has been read, and the state updates
+        // S^i^T += V^T K~i (which wait only for the state warps' rescale); the other issues everything that
+        // accumulates into the output tile.
         if (lane == 0) {
             prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-            auto load_tile = [&](int c) {
-                const int s = c & 1;
-                uint8_t* st = tiles + s * STAGE_BYTES;
-                const int t = t0 + c * C;
-                mbar_arrive_expect_tx(&sh.full[s], 6 * 8192);
-                tma_load_3d(st + OFF_Q, &map_q, &sh.full[s], 0, h, t);
-                tma_load_3d(st + OFF_Q + 8192, &map_q, &sh.full[s], 64, h, t);
-                tma_load_3d(st + OFF_K, &map_k, &sh.full[s], 0, h, t);
-                tma_load_3d(st + OFF_K + 8192, &map_k, &sh.full[s], 64, h, t);
-                tma_load_3d(st + OFF_V, &map_v, &sh.full[s], 0, h, t);
-                tma_load_3d(st + OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
-                if (c + 2 < nc) {   // pull the tile after next into L2 while this one is in flight
-                    const int t2 = t + 2 * C;
-                    tma_prefetch_3d(&map_q, 0, h, t2); tma_prefetch_3d(&map_q, 64, h, t2);
-                    tma_prefetch_3d(&map_k, 0, h, t2); tma_prefetch_3d(&map_k, 64, h, t2);
-                    tma_prefetch_3d(&map_v, 0, h, t2); tma_prefetch_3d(&map_v, 64, h, t2);
-                }
-            };
             const uint32_t sa = smem_u32(tiles);
+            constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
             constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4);
+            const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dk0 = smem_desc_sw128(sa + OFF_K, 16, 1024);
             const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
-            // iterations -2 and -1 only start the first two loads (one copy of the load code)
+            // iterations -2 and -1 only start the first two loads and the first scores
 #pragma unroll 1
             for (int c = -2; c < nc; ++c) {
                 const int s = c & 1;
                 const uint64_t so = (uint64_t)s * STAGE_STEP;
-                if (c >= 0) WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
-#pragma unroll 1
-                for (int i = 0; i < 2 && c >= 0; ++i) {
-                    WAITP(1, &sh.s_ready[i], c & 1);    // fp32 state i has been rescaled
+                if (c >= -1 && c + 1 < nc) {
+                    // P_{c+1}: K-major operands, four 32-byte k-steps inside a 64-element block, the next block 8 KB further
+                    WAITP(3, &sh.full[s ^ 1], ((c + 1) >> 1) & 1);
+                    if (c >= 0) WAITP(4, &sh.p_free, c & 1);            // every tile warp has seen P_c
                     tc_fence_after();
-                    const uint64_t a = dv0 + so, b = dkn0 + so + (uint64_t)(i * (16384 >> 4));
-                    { TLW_BEGIN;
+                    const uint64_t sn = (uint64_t)(s ^ 1) * STAGE_STEP;
+                    TLW_BEGIN;
+#pragma unroll 1
+                    for (int blk = 0; blk < 2; ++blk) {
+                        const uint64_t a = dq0 + sn + (uint64_t)(512 * blk), b = dk0 + sn + (uint64_t)(512 * blk);
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S + 128 * i, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
-                    tc_commit(&sh.u_full[i]);
-                    TLW_END(3); }
+                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_P, a + (uint64_t)(2 * kk), b + (uint64_t)(2 * kk), ID_P, (blk | kk) ? 1u : 0u);
+                    }
+                    tc_commit(&sh.p_full[0]);
+                    TLW_END(5);
+                    TL(1, c + 1, 7);
                 }
-                if (c >= 0) tc_commit(&sh.empty[s]);
-                TL(0, c, 5);
+                if (c >= 0) {
+                    WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
+#pragma unroll 1
+                    for (int i = 0; i < 2; ++i) {
+                        WAITP(1, &sh.s_ready[i], c & 1);    // fp32 state i has been rescaled
+                        tc_fence_after();
+                        const uint64_t a = dv0 + so, b = dkn0 + so + (uint64_t)(i * (16384 >> 4));
+                        TLW_BEGIN;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S + 128 * i, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
+                        tc_commit(&sh.u_full[i]);
+                        TLW_END(6);
+                    }
+                    tc_commit(&sh.empty[s]);
+                    TL(0, c, 5);
+                }
                 if (c + 2 < nc) {
                     if (c >= 0) WAITP(2, &sh.empty[s], (c >> 1) & 1);   // both issuers' MMAs on this stage are done
                     TL(0, c + 2, 0);
-                    { TLW_BEGIN; load_tile(c + 2); TLW_END(4); }
+                    TLW_BEGIN;
+                    uint8_t* st = tiles + s * STAGE_BYTES;
+                    const int t = t0 + (c + 2) * C;
+                    mbar_arrive_expect_tx(&sh.full[s], 6 * 8192);
+                    tma_load_4d(st + OFF_Q, &map_q, &sh.full[s], 0, t, 0, h);
+                    tma_load_4d(st + OFF_K, &map_k, &sh.full[s], 0, t, 0, h);
+                    tma_load_4d(st + OFF_V, &map_v, &sh.full[s], 0, t, 0, h);
+                    if (c + 4 < nc) {   // pull the tile after next into L2 while this one is in flight
+                        const int t2 = t + 2 * C;
+                        tma_prefetch_4d(&map_q, 0, t2, 0, h); tma_prefetch_4d(&map_k, 0, t2, 0, h); tma_prefetch_4d(&map_v, 0, t2, 0, h);
+                    }
+                    TLW_END(7);
                 }
             }
             TL_DUMP(0);
         }
     } else if (warp == WARP_MMA) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ MMA issuer of the output tile
+        // O^T = V^T P~^T + S1^T Q~1^T + S2^T Q~2^T : the first part does not need the states; each state has its own
+        // hand-off, so the bf16 copy of one runs under the MMAs of the other.  Groups of four MMAs with compile-time
+        // operand steps cost about half the issue time of a rolled loop.
         if (lane == 0) {
             const uint32_t sa = smem_u32(tiles);
-            constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OS = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OV = idesc_bf16(128, 64, 1, 0);
-            // Descriptors of stage 0; stage 1 and the k-steps are reached by adding constants to the address field.
             constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4), PT_STEP = (uint64_t)(8192 >> 4);
-            const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dk0 = smem_desc_sw128(sa + OFF_K, 16, 1024);
-            const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024);
+            const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024);
             const uint64_t dp0 = smem_desc_sw128(sa + OFF_PT, 16, 1024);
-            // One thread issues every MMA of the CTA.  Groups of four with compile-time operand steps cost about 45
-            // cycles per issue (a rolled loop about 80), which keeps the issue rate above the tensor pipe's.
-            auto run_ss4 = [&](uint32_t d, uint64_t a, uint64_t b, auto astep, auto bstep, uint32_t idesc, uint32_t acc) {
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ss(d, a + (uint64_t)(kk * decltype(astep)::value), b + (uint64_t)(kk * decltype(bstep)::value), idesc, kk > 0 ? 1u : acc);
-            };
-            auto run_ts4 = [&](uint32_t d, uint32_t a_tmem, uint64_t b, uint32_t idesc) {
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ts(d, a_tmem + 8 * kk, b + (uint64_t)(2 * kk), idesc, 1);
-            };
-            using S2 = std::integral_constant<int, 2>;
-            using S128 = std::integral_constant<int, 128>;
-            auto issue_p = [&](int c) {
-                const uint64_t so = (uint64_t)(c & 1) * STAGE_STEP;
-                // K-major operands: four 32-byte k-steps inside a 64-element block, then the next block 8 KB further
 #pragma unroll 1
-                for (int blk = 0; blk < 2; ++blk)
-                    run_ss4(tb + COL_P, dq0 + so + (uint64_t)(512 * blk), dk0 + so + (uint64_t)(512 * blk), S2{}, S2{}, ID_P, (uint32_t)blk);
-                tc_commit(&sh.p_full[0]);
-            };
-            mbar_wait(&sh.full[0], 0, abortp, p.status);
-            tc_fence_after();
-            issue_p(0);
             for (int c = 0; c < nc; ++c) {
                 const int s = c & 1;
                 const uint64_t so = (uint64_t)s * STAGE_STEP;
-                // Scores of the next chunk go out as soon as its tile has landed and every tile warp has seen P_c:
-                // polled between the MMA groups of this chunk so the tile warps can start on the next one early.
-                // stage: 0 V part (waits for the operands), 2/3 state parts, 6 done
-                bool p_next_done = c + 1 >= nc;
-                int stage = 0;
-#pragma unroll 1
-                for (uint32_t spin = 0; spin < 40000000u && !(p_next_done && stage == 6); ++spin) {
-#ifdef DSLA_TIMELINE
-                    const long long tl_a = clock64();
-                    const int tl_stage = stage; const bool tl_p = p_next_done;
-#endif
-                    if (!p_next_done && mbar_test_wait(&sh.full[(c + 1) & 1], ((c + 1) >> 1) & 1) && mbar_test_wait(&sh.p_free, c & 1)) {
-                        tc_fence_after();
-                        { TLW_BEGIN; issue_p(c + 1); TLW_END(4); }
-                        p_next_done = true;
-                        TL(1, c + 1, 7);
-                    }
-                    if (stage == 0) {
-                        if (mbar_test_wait(&sh.prep_ready[0], c & 1) && (c == 0 || mbar_test_wait(&sh.o_free, (c - 1) & 1))) {
-                            TL(1, c, 1);
-                            tc_fence_after();
-                            // O^T = V^T P~^T + S1^T Q~1^T + S2^T Q~2^T ; the first part does not need the states
-                            { TLW_BEGIN; run_ss4(tb + COL_O, dv0 + so, dp0 + (uint64_t)s * PT_STEP, S128{}, S2{}, ID_OV, 0); TLW_END(2); }
-                            stage = 2;
-                        }
-                    } else if (stage == 2 || stage == 3) {
-                        // each state has its own hand-offs: the copy / rescale pass of one runs under the MMAs of the other
-                        const int i = stage - 2;
-                        if (mbar_test_wait(&sh.sb_ready[i], c & 1)) {
-                            if (i == 0) TL(1, c, 3);
-                            tc_fence_after();
-                            const uint64_t dq = dq0 + so + (uint64_t)(i * (16384 >> 4));
-                            { TLW_BEGIN;
-                            run_ts4(tb + COL_O, tb + COL_SB + 64 * i, dq, ID_OS);
-                            run_ts4(tb + COL_O, tb + COL_SB + 64 * i + 32, dq + 512, ID_OS);
-                            TLW_END(3); }
-                            if (i == 1) { TLW_BEGIN; tc_commit(&sh.o_full[0]); tc_commit(&sh.empty[s]); TLW_END(5); TL(1, c, 6); }
-                            stage = i == 0 ? 3 : 6;
-                        }
-                    }
-#ifdef DSLA_TIMELINE
-                    if (tl_stage != stage || tl_p != p_next_done) TLACC(1, clock64() - tl_a); else TLACC(0, clock64() - tl_a);
-#endif
-                    if ((spin & 4095u) == 4095u && *abortp) break;
+                WAITP(0, &sh.prep_ready[0], c & 1);
+                if (c > 0) WAITP(1, &sh.o_free, (c - 1) & 1);
+                TL(1, c, 1);
+                tc_fence_after();
+                {
+                    TLW_BEGIN;
+                    const uint64_t a = dv0 + so, b = dp0 + (uint64_t)s * PT_STEP;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, a + (uint64_t)(kk * 128), b + (uint64_t)(2 * kk), ID_OV, kk ? 1u : 0u);
+                    TLW_END(4);
                 }
-                if (!(p_next_done && stage == 6) && !*abortp) { *abortp = 1; atomicExch(p.status, 5); }
+#pragma unroll 1
+                for (int i = 0; i < 2; ++i) {
+                    WAITP(2, &sh.sb_ready[i], c & 1);
+                    if (i == 0) TL(1, c, 3);
+                    tc_fence_after();
+                    TLW_BEGIN;
+                    const uint64_t dq = dq0 + so + (uint64_t)(i * (16384 >> 4));
+                    const uint32_t at = tb + COL_SB + 64 * i;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_O, at + 8 * kk, dq + (uint64_t)(2 * kk), ID_OS, 1);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_O, at + 32 + 8 * kk, dq + 512 + (uint64_t)(2 * kk), ID_OS, 1);
+                    TLW_END(5);
+                }
+                tc_commit(&sh.o_full[0]);
+                tc_commit(&sh.empty[s]);
+                TL(1, c, 6);
             }
             TL_DUMP(1);
         }
@@ -500,16 +474,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (warp == 6 && lane == 0) TL_DUMP(3);
     } else if (warp >= GATE_W0) {
         // ------------------------------------------------------------------ gate warps 18,19
-        // Running products of gates down the rows give the decay mask without logs or exps (a zero gate
-        // gives an exact zero): M[j][s] = W1 d_1(j,s) + W2 d_2(j,s), d_i(j,s) = prod_{t=s+1..j} g^i_t, 0 for s > j.
-        // Warp 18 owns columns 0..31 (rows 0..31 from 1, rows 32..63 continuing from the product to row 31),
-        // warp 19 columns 32..63 (rows 32..63).  The per-token factors come from warp-wide product scans:
-        //   w^i_s    = prod_{t > s} g^i_t                     (decay to the end of the chunk)
-        //   rowf^i_j = W_i prod_{t <= j} g^i_t                (decay from the chunk start through token j)
+        // Everything the chunk needs from the gates comes from the cumulative log-gates
+        //     L^i_j = sum_{t <= j} log2 g^i_t        (inclusive, from the chunk start; a zero gate counts as -200,
+        //                                             so any product that contains one flushes to an exact zero)
+        // through independent exponentials (no serial chains):
+        //   M[j][s]  = W1 2^(L1_j - L1_s) + W2 2^(L2_j - L2_s)  for s <= j, else 0      (decay mask)
+        //   rowf^i_j = W_i 2^(L^i_j)                  (decay from the chunk start through token j)
+        //   w^i_s    = 2^(L^i_last - L^i_s)           (decay from token s to the end of the chunk)
+        // Lane l holds tokens l and l + 32.  Warp 18 writes the triangle of rows/columns 0..31, warp 19 the
+        // triangle of 32..63; the full block (rows 32..63, columns 0..31) factors through token 31,
+        // 2^(L_j - L_31) 2^(L_31 - L_s) with both factors <= 1, and is split between the two warps.
         const int gw = warp - GATE_W0;
         const float gam = p.gamma[h];
         const float W1 = gam * p.scale, W2 = (1.f - gam) * p.scale;
-        // each warp keeps all 64 gate pairs of the chunk in registers: lane l holds tokens l and l + 32
         auto fetch = [&](int c, float2& lo, float2& hi2) {
             const int j = c * C + lane;
             const bool in = c < nc;
@@ -526,51 +503,44 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             __nv_bfloat16* Mm = reinterpret_cast<__nv_bfloat16*>(tiles + OFF_MASK + s * MASK_BYTES);
             const float2 glo = nlo, ghi = nhi;
             fetch(c + 1, nlo, nhi);
+            TLT(tlg0);
+            float l1a = warp_prefix_sum(lg2_gate(glo.x), lane), l2a = warp_prefix_sum(lg2_gate(glo.y), lane);
+            float l1b = warp_prefix_sum(lg2_gate(ghi.x), lane), l2b = warp_prefix_sum(lg2_gate(ghi.y), lane);
+            const float mid1 = __shfl_sync(0xffffffffu, l1a, 31), mid2 = __shfl_sync(0xffffffffu, l2a, 31);   // L at token 31
+            l1b += mid1; l2b += mid2;
+            const float end1 = __shfl_sync(0xffffffffu, l1b, 31), end2 = __shfl_sync(0xffffffffu, l2b, 31);   // L at token 63
             if (c >= 2) WAITP(0, &sh.m_free[s], ((c >> 1) - 1) & 1);
             if (warp == GATE_W0 && lane == 0) TL(0, c, 1);
-            TLT(tlg0);
-            // suffix products of the lower half for both states (start values of rows 32..63 in columns 0..31)
-            const float slx = warp_suffix_prod(glo.x, lane), sly = warp_suffix_prod(glo.y, lane);
             {
-                const float xl = gw == 0 ? glo.x : glo.y, xh = gw == 0 ? ghi.x : ghi.y;   // this warp's state
+                // per-token factors of this warp's state
+                const float la = gw == 0 ? l1a : l2a, lb = gw == 0 ? l1b : l2b, le = gw == 0 ? end1 : end2;
                 const float Wi = gw == 0 ? W1 : W2;
-                const float sl_in = gw == 0 ? slx : sly;
-                const float pl = warp_prefix_prod(xl, lane), ph0 = warp_prefix_prod(xh, lane);
-                const float tot_lo = __shfl_sync(0xffffffffu, pl, 31);
-                const float sh_in = warp_suffix_prod(xh, lane);
-                const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0);
-                float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
-                if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
                 const int valid = min(C, sq.len - tok0 - c * C);
-                gs.rowf[gw][lane] = dup_bf16(Wi * pl);
-                gs.rowf[gw][lane + 32] = dup_bf16(Wi * tot_lo * ph0);
+                gs.rowf[gw][lane] = dup_bf16(Wi * ex2(la));
+                gs.rowf[gw][lane + 32] = dup_bf16(Wi * ex2(lb));
                 // rows past the end of the sequence carry no weight in the state update
-                gs.w[gw][lane] = dup_bf16(lane < valid ? sl_ex * tot_hi : 0.f);
-                gs.w[gw][lane + 32] = dup_bf16(lane + 32 < valid ? sh_ex : 0.f);
+                gs.w[gw][lane] = dup_bf16(lane < valid ? ex2(le - la) : 0.f);
+                gs.w[gw][lane + 32] = dup_bf16(lane + 32 < valid ? ex2(le - lb) : 0.f);
             }
             TLT(tlg1); TLACC(1, tlg1 - tlg0);
-            if (gw == 0) {
-                float ex = __shfl_down_sync(0xffffffffu, slx, 1), ey = __shfl_down_sync(0xffffffffu, sly, 1);
-                if (lane == 31) { ex = 1.f; ey = 1.f; }
-                float a1 = 1.f, a2 = 1.f, b1 = ex, b2 = ey;     // chains: rows 0..31 (triangle) and rows 32..63 (full)
-                __nv_bfloat16* mcol = Mm + lane;
-#pragma unroll 4
+            {
+                // triangle block of this warp: rows and columns 32 gw .. 32 gw + 31, this lane = column
+                const float x1 = gw == 0 ? l1a : l1b, x2 = gw == 0 ? l2a : l2b;
+                __nv_bfloat16* mcol = Mm + (32 * gw) * MASK_PITCH + 32 * gw + lane;
+#pragma unroll 8
                 for (int jj = 0; jj < 32; ++jj) {
-                    const float gxa = __shfl_sync(0xffffffffu, glo.x, jj), gya = __shfl_sync(0xffffffffu, glo.y, jj);
-                    const float gxb = __shfl_sync(0xffffffffu, ghi.x, jj), gyb = __shfl_sync(0xffffffffu, ghi.y, jj);
-                    if (jj > lane) { a1 *= gxa; a2 *= gya; }
-                    b1 *= gxb; b2 *= gyb;
-                    mcol[jj * MASK_PITCH] = __float2bfloat16_rn(jj >= lane ? fmaf(W2, a2, W1 * a1) : 0.f);
-                    mcol[(32 + jj) * MASK_PITCH] = __float2bfloat16_rn(fmaf(W2, b2, W1 * b1));
+                    const float r1 = __shfl_sync(0xffffffffu, x1, jj), r2 = __shfl_sync(0xffffffffu, x2, jj);
+                    const float m = fmaf(W2, ex2(r2 - x2), W1 * ex2(r1 - x1));
+                    mcol[jj * MASK_PITCH] = __float2bfloat16_rn(jj >= lane ? m : 0.f);
                 }
-            } else {
-                float a1 = 1.f, a2 = 1.f;
-                __nv_bfloat16* mcol = Mm + 32 * MASK_PITCH + 32 + lane;
-#pragma unroll 4
-                for (int jj = 0; jj < 32; ++jj) {
-                    const float gx = __shfl_sync(0xffffffffu, ghi.x, jj), gy = __shfl_sync(0xffffffffu, ghi.y, jj);
-                    if (jj > lane) { a1 *= gx; a2 *= gy; }
-                    mcol[jj * MASK_PITCH] = __float2bfloat16_rn(jj >= lane ? fmaf(W2, a2, W1 * a1) : 0.f);
+                // full block: rows 32 + 16 gw .. + 15, columns 0..31
+                const float f1 = ex2(mid1 - l1a), f2 = ex2(mid2 - l2a);                 // column factors (token s -> 31)
+                const float e1 = W1 * ex2(l1b - mid1), e2 = W2 * ex2(l2b - mid2);       // row factors (31 -> token 32 + lane)
+                __nv_bfloat16* mrow = Mm + (32 + 16 * gw) * MASK_PITCH + lane;
+#pragma unroll 8
+                for (int jj = 0; jj < 16; ++jj) {
+                    const float a1 = __shfl_sync(0xffffffffu, e1, 16 * gw + jj), a2 = __shfl_sync(0xffffffffu, e2, 16 * gw + jj);
+                    mrow[jj * MASK_PITCH] = __float2bfloat16_rn(fmaf(a2, f2, a1 * f1));
                 }
             }
             TLACC(2, clock64() - tlg1);
@@ -749,10 +719,8 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                 uint8_t* st = tiles + s * SUM_STAGE_BYTES;
                 const int t = t0 + (nc - 1 - it) * C;
                 mbar_arrive_expect_tx(&sh.full[s], 4 * 8192);
-                tma_load_3d(st, &map_k, &sh.full[s], 0, h, t);
-                tma_load_3d(st + 8192, &map_k, &sh.full[s], 64, h, t);
-                tma_load_3d(st + SUM_OFF_V, &map_v, &sh.full[s], 0, h, t);
-                tma_load_3d(st + SUM_OFF_V + 8192, &map_v, &sh.full[s], 64, h, t);
+                tma_load_4d(st, &map_k, &sh.full[s], 0, t, 0, h);
+                tma_load_4d(st + SUM_OFF_V, &map_v, &sh.full[s], 0, t, 0, h);
             }
         }
     } else if (warp == 9) {
@@ -851,14 +819,17 @@ EncodeFn get_encode() {
 }
 
 // Tensor [T_total][H][128] bf16 viewed as (d, H, T); a box is 64 d-elements (128 B) x 1 head x 64 tokens.
+// [T_total, H, 128] bf16 seen as (x: 64 elements, t, half: the two 64-element halves of a row, h) so that one
+// copy of box {64, 64 tokens, 2, 1} lands as two consecutive 8 KB tiles [half][token][64], each in the 128-byte
+// swizzle the MMA descriptors expect.
 bool make_map(CUtensorMap* m, const void* base, int T_total, int H) {
     EncodeFn fn = get_encode();
     if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T_total};
-    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2};
-    cuuint32_t box[3] = {64, 1, 64};
-    cuuint32_t es[3] = {1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+    cuuint64_t dims[4] = {64, (cuuint64_t)T_total, 2, (cuuint64_t)H};
+    cuuint64_t strides[3] = {(cuuint64_t)H * D * 2, 128, (cuuint64_t)D * 2};
+    cuuint32_t box[4] = {64, 64, 2, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
