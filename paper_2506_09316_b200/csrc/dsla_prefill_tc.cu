@@ -54,19 +54,28 @@ constexpr uint32_t COL_P = 448;    // P, 64 columns (lanes 0..63 meaningful)
 constexpr size_t SUMMARY_STRIDE = 2 * D * D * sizeof(float) + 256;  // U (both states) + A[2], padded
 
 #ifdef DSLA_TIMELINE
-__device__ long long* g_timeline = nullptr;   // [role 4][chunk 64][event 8]
+__device__ long long* g_timeline = nullptr;   // [role 6][chunk 64][event 8], then per-CTA start/end times, then counters
 __device__ int g_timeline_block = 0;
 #define TL(role, c, ev) do { if (tlp && (unsigned)(c) < 64u) tlp[((role) * 64 + (c)) * 8 + (ev)] = clock64(); } while (0)
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#ifdef DSLA_TLW   // per-thread wait / section counters on top of the event timeline (costs ~20 registers)
 #define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr; \
     long long tl_w[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; const long long tl_t0 = clock64()
-// wait with the cycles it took added to this thread's counter `tag`; TL_DUMP writes a role's counters and its lifetime
 #define WAITP(tag, bar, ph) do { const long long _a = clock64(); mbar_wait(bar, ph, abortp, p.status); tl_w[tag] += clock64() - _a; } while (0)
 #define TLT(var) const long long var = clock64()
 #define TLACC(tag, expr) tl_w[tag] += (expr)
 #define TLW_BEGIN const long long _tlb = clock64()
 #define TLW_END(tag) tl_w[tag] += clock64() - _tlb
-#define TL_DUMP(role) do { if (tlp) { for (int _k = 0; _k < 10; ++_k) tlp[2700 + 12 * (role) + _k] = tl_w[_k]; tlp[2700 + 12 * (role) + 10] = clock64() - tl_t0; } } while (0)
+#define TL_DUMP(role) do { if (tlp) { for (int _k = 0; _k < 10; ++_k) tlp[3800 + 12 * (role) + _k] = tl_w[_k]; tlp[3800 + 12 * (role) + 10] = clock64() - tl_t0; } } while (0)
+#else
+#define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr
+#define WAITP(tag, bar, ph) mbar_wait(bar, ph, abortp, p.status)
+#define TLT(var) do { } while (0)
+#define TLACC(tag, expr) do { } while (0)
+#define TLW_BEGIN do { } while (0)
+#define TLW_END(tag) do { } while (0)
+#define TL_DUMP(role) do { } while (0)
+#endif
 #else
 #define WAITP(tag, bar, ph) mbar_wait(bar, ph, abortp, p.status)
 #define TLT(var) do { } while (0)
@@ -214,7 +223,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     TL_INIT;
     if (tid == 0) TL(0, 63, 6);
 #ifdef DSLA_TIMELINE
-    if (tid == 0 && g_timeline) g_timeline[2048 + 4 * blockIdx.x] = gtime();
+    if (tid == 0 && g_timeline) g_timeline[3072 + 4 * blockIdx.x] = gtime();
 #endif
 
     if (tid == 0) {
@@ -259,6 +268,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     // P_{c+1}: K-major operands, four 32-byte k-steps inside a 64-element block, the next block 8 KB further
                     WAITP(3, &sh.full[s ^ 1], ((c + 1) >> 1) & 1);
                     if (c >= 0) WAITP(4, &sh.p_free, c & 1);            // every tile warp has seen P_c
+                    TL(4, c + 1, 1);
                     tc_fence_after();
                     const uint64_t sn = (uint64_t)(s ^ 1) * STAGE_STEP;
                     TLW_BEGIN;
@@ -270,13 +280,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     }
                     tc_commit(&sh.p_full[0]);
                     TLW_END(5);
-                    TL(1, c + 1, 7);
+                    TL(4, c + 1, 2);
                 }
                 if (c >= 0) {
                     WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
+                    TL(4, c, 3);
 #pragma unroll 1
                     for (int i = 0; i < 2; ++i) {
                         WAITP(1, &sh.s_ready[i], c & 1);    // fp32 state i has been rescaled
+                        TL(4, c, 4 + i);
                         tc_fence_after();
                         const uint64_t a = dv0 + so, b = dkn0 + so + (uint64_t)(i * (16384 >> 4));
                         TLW_BEGIN;
@@ -286,11 +298,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         TLW_END(6);
                     }
                     tc_commit(&sh.empty[s]);
-                    TL(0, c, 5);
+                    TL(4, c, 6);
                 }
                 if (c + 2 < nc) {
                     if (c >= 0) WAITP(2, &sh.empty[s], (c >> 1) & 1);   // both issuers' MMAs on this stage are done
-                    TL(0, c + 2, 0);
+                    if (c >= 0) TL(4, c, 7);
                     TLW_BEGIN;
                     uint8_t* st = tiles + s * STAGE_BYTES;
                     const int t = t0 + (c + 2) * C;
@@ -303,6 +315,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         tma_prefetch_4d(&map_q, 0, t2, 0, h); tma_prefetch_4d(&map_k, 0, t2, 0, h); tma_prefetch_4d(&map_v, 0, t2, 0, h);
                     }
                     TLW_END(7);
+                    TL(4, c + 2, 0);
                 }
             }
             TL_DUMP(0);
@@ -323,6 +336,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             for (int c = 0; c < nc; ++c) {
                 const int s = c & 1;
                 const uint64_t so = (uint64_t)s * STAGE_STEP;
+                TL(1, c, 0);
                 WAITP(0, &sh.prep_ready[0], c & 1);
                 if (c > 0) WAITP(1, &sh.o_free, (c - 1) & 1);
                 TL(1, c, 1);
@@ -333,11 +347,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, a + (uint64_t)(kk * 128), b + (uint64_t)(2 * kk), ID_OV, kk ? 1u : 0u);
                     TLW_END(4);
+                    TL(1, c, 2);
                 }
 #pragma unroll 1
                 for (int i = 0; i < 2; ++i) {
                     WAITP(2, &sh.sb_ready[i], c & 1);
-                    if (i == 0) TL(1, c, 3);
+                    TL(1, c, 3 + i);
                     tc_fence_after();
                     TLW_BEGIN;
                     const uint64_t dq = dq0 + so + (uint64_t)(i * (16384 >> 4));
@@ -368,6 +383,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // bytes (two full sectors), so the outputs go straight from registers to global memory
         auto outputs = [&](int c) {
             WAITP(0, &sh.o_full[0], c & 1);
+            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 3);
             tc_fence_after();
             TLT(tlo0);
             uint32_t r[32];
@@ -376,7 +392,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             TLT(tlo1); TLACC(5, tlo1 - tlo0);
             __syncwarp();
             if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
-            if (warp == 4 && lane == 0) TL(2, c, 4);
+            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 4);
             const int valid = min(C, sq.len - tok0 - c * C) - 32 * half;     // tokens of this warp's half that exist
             __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * half) * p.H + h) * D + 32 * q + lane;
             const size_t row = (size_t)p.H * D;
@@ -393,7 +409,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
             }
             TLACC(6, clock64() - tlo1);
-            if (warp == 4 && lane == 0) TL(2, c, 5);
+            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 5);
         };
 
         // Iteration c builds the operands of chunk c (c < nc) and stores the outputs of chunk c-1 (c > 0); the
@@ -403,7 +419,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             GateSmem& gs = sh.gs[s];
             uint8_t* st = tiles + s * STAGE_BYTES;
             const uint8_t* Mm = tiles + OFF_MASK + s * MASK_BYTES;
-            if (warp == 4 && lane == 0) TL(2, c, 0);
+            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 0);
             bool out_done = c == 0;
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
@@ -416,7 +432,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 WAITP(3, &sh.full[s], (c >> 1) & 1);
                 WAITP(4, &sh.p_full[0], c & 1);   // P ready; the MMA is also done reading raw Q, K
                 tc_fence_after();
-                if (warp == 4 && lane == 0) TL(2, c, 1);
+                if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 1);
                 TLT(tlm0);
                 if (q >= 2 && lane == 0) mbar_arrive(&sh.p_free);   // these warps do not read P; they only had to see this phase
                 if (q < 2) {
@@ -467,7 +483,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.prep_ready[0]); mbar_arrive(&sh.m_free[s]); }
-                if (warp == 4 && lane == 0) TL(2, c, 2);
+                if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 2);
             }
         }
         if (warp == 4 && lane == 0) TL_DUMP(2);
@@ -659,7 +675,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     __syncthreads();
     if (tid == 0) TL(0, 63, 7);
 #ifdef DSLA_TIMELINE
-    if (tid == 0 && g_timeline) g_timeline[2048 + 4 * blockIdx.x + 1] = gtime();
+    if (tid == 0 && g_timeline) g_timeline[3072 + 4 * blockIdx.x + 1] = gtime();
 #endif
     if (warp == WARP_MMA) tmem_dealloc(tb, 512);
 }
