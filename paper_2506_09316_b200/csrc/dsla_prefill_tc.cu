@@ -91,7 +91,9 @@ struct TcParams {
     PrefillParams p;
     float* ws;          // summaries: [(n*H + h)*nseg + g] -> {U[2][D][D], A[2]}
     int nseg;           // segments per sequence (grid dimension)
-    int cps;            // chunks per segment
+    int cps;            // chunks per segment (mean)
+    int skew8;          // eighths of a chunk by which consecutive segments get shorter (later segments start later: they
+                        // first fold the summaries of all earlier segments into their initial state)
     const int* order;   // sequences by descending length (longest first), or nullptr for index order
 };
 
@@ -136,16 +138,22 @@ struct SeqInfo {
     int t_begin, len, slot, nchunks, c_begin, c_end, last_seg;
 };
 
-__device__ __forceinline__ SeqInfo seq_info(const PrefillParams& p, int n, int g, int cps) {
+// First chunk of segment g: equal parts of cps chunks, shifted so that segment g is about skew8 (nseg - 2g - 1) / 8
+// chunks longer than the mean.  seg_begin(0) = 0 and seg_begin(nseg) = nseg cps.
+__host__ __device__ __forceinline__ int seg_begin(int g, int nseg, int cps, int skew8) { return g * cps + (skew8 * g * (nseg - g)) / 8; }
+
+__device__ __forceinline__ SeqInfo seq_info(const PrefillParams& p, int n, int g, int nseg, int cps, int skew8) {
     SeqInfo s;
     s.t_begin = p.cu_seqlens ? p.cu_seqlens[n] : n * p.T;
     const int t_end = p.cu_seqlens ? p.cu_seqlens[n + 1] : (n + 1) * p.T;
     s.len = t_end - s.t_begin;
     s.slot = p.slots ? p.slots[n] : n;
     s.nchunks = (s.len + C - 1) / C;
-    s.c_begin = g * cps;
-    s.c_end = min(s.nchunks, (g + 1) * cps);
-    s.last_seg = s.nchunks > 0 ? (s.nchunks - 1) / cps : 0;
+    s.c_begin = seg_begin(g, nseg, cps, skew8);
+    s.c_end = min(s.nchunks, seg_begin(g + 1, nseg, cps, skew8));
+    s.last_seg = 0;     // the last segment that holds a chunk of this sequence
+    for (int j = 1; j < nseg; ++j)
+        if (seg_begin(j, nseg, cps, skew8) < s.nchunks) s.last_seg = j;
     return s;
 }
 
@@ -207,7 +215,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int h = (blockIdx.x / tp.nseg) % p.H;
     const int rank = blockIdx.x / (tp.nseg * p.H);
     const int n = tp.order ? tp.order[rank] : rank;
-    const SeqInfo sq = seq_info(p, n, g, tp.cps);
+    const SeqInfo sq = seq_info(p, n, g, tp.nseg, tp.cps, tp.skew8);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
     float* slot1 = p.state + (((size_t)sq.slot * 2) * p.H + h) * (size_t)(D * D);
     const size_t state_stride = (size_t)p.H * D * D;
@@ -594,12 +602,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const float2 gp_next = gate_pair(c + 1);
             if (warp == 12 && lane == 0) TL(3, c, 0);
             if (c == 0) {
+                // With programmatic dependent launch this grid may start while the summary grid is still running;
+                // everything up to here (and all of chunk 0's operand work in the other warps) is independent of it.
+                if (g > 0 && tp.ws) asm volatile("griddepcontrol.wait;" ::: "memory");
                 init_state_pass(slot1 + (size_t)hi * state_stride, p.use_initial_state,
                                 tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, hi, v, a, s_addr, sb_addr);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.sb_ready[hi]); mbar_arrive(&sh.s_ready[hi]); }
+#ifdef DSLA_TIMELINE
+                if (warp == 12 && lane == 0 && g_timeline) g_timeline[3072 + 4 * blockIdx.x + 2] = gtime();
+#endif
                 a_next = warp_prod(gp_next);
                 continue;
             }
@@ -609,8 +623,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (warp == 12 && lane == 0) TL(3, c, 1);
             if (warp == 16 && lane == 0) TL(3, c, 4);
             TLT(tls0);
-            // ---- A. bf16 copy of S_c: the readout of chunk c waits for this
+            // ---- one pass over the state (TMEM -> registers once): the bf16 copy of S_{c-1} that the readout of chunk c
+            // multiplies, and a_c S_{c-1} in place, onto which the update MMA of chunk c accumulates
             {
+                const float2 a2 = make_float2(a, a);
                 uint32_t r0[32], r1[32];
                 tmem_ld32(s_addr, r0);
                 tmem_ld32(s_addr + 32, r1);
@@ -624,25 +640,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                     for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(__uint_as_float(r1[2 * k]), __uint_as_float(r1[2 * k + 1]));
                     tmem_st16(sb_addr + 32 * half + 16, pk);
-                    if (half == 0) { tmem_ld32(s_addr + 64, r0); tmem_ld32(s_addr + 96, r1); }
-                }
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.sb_ready[hi]);
-            }
-            if (warp == 12 && lane == 0) TL(3, c, 2);
-            if (warp == 16 && lane == 0) TL(3, c, 5);
-            TLT(tls1); TLACC(2, tls1 - tls0);
-            // ---- B. S <- a_c S: the state update of chunk c waits for this (it runs behind the readout MMAs)
-            {
-                const float2 a2 = make_float2(a, a);
-                uint32_t r0[32], r1[32];
-                tmem_ld32(s_addr, r0);
-                tmem_ld32(s_addr + 32, r1);
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    tc_wait_ld();
 #pragma unroll
                     for (int k = 0; k < 32; k += 2) {
                         const float2 y0 = __fmul2_rn(make_float2(__uint_as_float(r0[k]), __uint_as_float(r0[k + 1])), a2);
@@ -657,8 +654,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.s_ready[hi]);
+                if (lane == 0) { mbar_arrive(&sh.sb_ready[hi]); mbar_arrive(&sh.s_ready[hi]); }
             }
+            if (warp == 12 && lane == 0) TL(3, c, 2);
+            if (warp == 16 && lane == 0) TL(3, c, 5);
+            TLT(tls1); TLACC(2, tls1 - tls0);
             TLACC(3, clock64() - tls1);
             a_next = warp_prod(gp_next);
             if (warp == 12 && lane == 0) TL(3, c, 3);
@@ -668,6 +668,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (warp == 16 && lane == 0) TL_DUMP(5);
         // ---- final states of this segment's last chunk
         mbar_wait(&sh.u_full[hi], (nc - 1) & 1, abortp, p.status);
+#ifdef DSLA_TIMELINE
+        if (warp == 12 && lane == 0 && g_timeline) g_timeline[3072 + 4 * blockIdx.x + 3] = gtime();
+#endif
         tc_fence_after();
         if (g == sq.last_seg) store_state(slot1 + (size_t)hi * state_stride, v, s_addr);
     }
@@ -697,12 +700,16 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     const PrefillParams& p = tp.p;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef DSLA_TIMELINE
+    if (threadIdx.x == 0 && g_timeline) g_timeline[4096 + 4 * blockIdx.x] = gtime();
+#endif
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main grid may be scheduled as SMs become free
     const int nsum = tp.nseg - 1;
     const int g = blockIdx.x % nsum;
     const int h = (blockIdx.x / nsum) % p.H;
     const int rank = blockIdx.x / (nsum * p.H);
     const int n = tp.order ? tp.order[rank] : rank;
-    const SeqInfo sq = seq_info(p, n, g, tp.cps);
+    const SeqInfo sq = seq_info(p, n, g, tp.nseg, tp.cps, tp.skew8);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
     if (sq.len <= 0 || g >= sq.last_seg) return;      // only segments that have a successor
     const int nc = sq.c_end - sq.c_begin;             // full chunks only (not the sequence's last segment)
@@ -791,6 +798,9 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             uint8_t* st = tiles + s * SUM_STAGE_BYTES;
             mbar_wait(&w_ready[s], u & 1, abortp, p.status);
             mbar_wait(&sh.full[s], u & 1, abortp, p.status);
+#ifdef DSLA_TIMELINE
+            if (tid == 0 && it == 0 && g_timeline) g_timeline[4096 + 4 * blockIdx.x + 2] = gtime();
+#endif
 #pragma unroll 2
             for (int m = 0; m < 4; ++m) {
                 const int idx = tid + SUM_NCOMPUTE * m;
@@ -806,11 +816,17 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             if (lane == 0) { mbar_arrive(&k_ready[s]); mbar_arrive(&w_free[s]); }
         }
         mbar_wait(&sh.u_full[0], 0, abortp, p.status);
+#ifdef DSLA_TIMELINE
+        if (tid == 0 && g_timeline) g_timeline[4096 + 4 * blockIdx.x + 3] = gtime();
+#endif
         tc_fence_after();
         store_state(out + (size_t)hi * D * D, 32 * q + lane, lane_addr + 128 * hi);
     }
     tc_fence_before();
     __syncthreads();
+#ifdef DSLA_TIMELINE
+    if (tid == 0 && g_timeline) g_timeline[4096 + 4 * blockIdx.x + 1] = gtime();
+#endif
     if (warp == 9) tmem_dealloc(tb, 256);
 }
 
@@ -873,7 +889,7 @@ __global__ void seq_order_kernel(const int32_t* __restrict__ cu, int N, int* __r
 
 bool wants_order(const dsla_prefill_args* a) { return a->cu_seqlens != nullptr && a->N > 1 && a->N <= ORDER_MAX_N; }
 
-void plan(const dsla_prefill_args* a, int* nseg, int* cps) {
+void plan(const dsla_prefill_args* a, int* nseg, int* cps, int* skew8) {
     const int max_chunks = (a->max_seqlen + C - 1) / C;
     const long long units = (long long)a->N * a->H;
     int ns = 1;
@@ -883,6 +899,10 @@ void plan(const dsla_prefill_args* a, int* nseg, int* cps) {
     if (max_chunks <= 0) ns = 1;
     *nseg = ns;
     *cps = max_chunks > 0 ? (max_chunks + ns - 1) / ns : 1;
+    // later segments fold more summaries into their initial state before they start (about 0.8 chunk times each):
+    // make consecutive segments 3/4 chunk shorter, as far as the shortest keeps at least three chunks
+    int sk = ns > 1 ? (8 * (*cps - 3)) / (ns - 1) : 0;
+    *skew8 = sk < 0 ? 0 : (sk > 3 ? 3 : sk);
 }
 
 }  // namespace
@@ -897,8 +917,8 @@ extern "C" int dsla_debug_set_timeline(long long* dev_ptr, int block) {
 bool prefill_tc_available() { return true; }
 
 size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a) {
-    int nseg, cps;
-    plan(a, &nseg, &cps);
+    int nseg, cps, skew8;
+    plan(a, &nseg, &cps, &skew8);
     const size_t summaries = nseg > 1 ? (size_t)a->N * a->H * nseg * SUMMARY_STRIDE : 0;     // a multiple of 256
     const size_t order = wants_order(a) ? (((size_t)a->N * sizeof(int) + 255) & ~(size_t)255) : 0;
     return summaries + order;
@@ -911,7 +931,7 @@ dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a
     }
     TcParams tp;
     tp.p = p;
-    plan(a, &tp.nseg, &tp.cps);
+    plan(a, &tp.nseg, &tp.cps, &tp.skew8);
     tp.ws = tp.nseg > 1 ? static_cast<float*>(a->workspace) : nullptr;
     tp.order = nullptr;
     if (wants_order(a)) {
@@ -933,7 +953,21 @@ dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a
         prefill_tc_summary_kernel<<<dim3((unsigned)(units * (tp.nseg - 1))), dim3(SUM_NTHREADS), SUM_SMEM_DYN, s>>>(mk, mv, tp);
         count_launch();
     }
-    prefill_tc_kernel<<<dim3((unsigned)(units * tp.nseg)), dim3(NTHREADS), SMEM_DYN, s>>>(mq, mk, mv, tp);
+    {
+        // Programmatic dependent launch after the summary grid: the main grid's prologue and the first chunk's
+        // operand work overlap the summary grid's tail; the state warps wait for it before they read the summaries.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(units * tp.nseg));
+        cfg.blockDim = dim3(NTHREADS);
+        cfg.dynamicSmemBytes = SMEM_DYN;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = tp.nseg > 1 ? 1 : 0;
+        if (cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, tp) != cudaSuccess) return DSLA_ERR_CUDA;
+    }
     count_launch();
     return cudaGetLastError() == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
 }
