@@ -263,7 +263,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);
-            constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
+            constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
             constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4);
             const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dk0 = smem_desc_sw128(sa + OFF_K, 16, 1024);
             const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
@@ -293,16 +293,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (c >= 0) {
                     WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
                     TL(4, c, 3);
-#pragma unroll 1
-                    for (int i = 0; i < 2; ++i) {
-                        WAITP(1, &sh.s_ready[i], c & 1);    // fp32 state i has been rescaled
-                        TL(4, c, 4 + i);
-                        tc_fence_after();
-                        const uint64_t a = dv0 + so, b = dkn0 + so + (uint64_t)(i * (16384 >> 4));
+                    // both states in one N = 256 MMA per k-step: [S1^T S2^T] += V^T [K~1 K~2] (the two K~ tiles and the two
+                    // fp32 states are adjacent), so V^T is read from shared memory once
+                    WAITP(1, &sh.s_ready[0], c & 1);        // fp32 states have been rescaled
+                    WAITP(1, &sh.s_ready[1], c & 1);
+                    TL(4, c, 5);
+                    tc_fence_after();
+                    {
+                        const uint64_t a = dv0 + so, b = dkn0 + so;
                         TLW_BEGIN;
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S + 128 * i, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
-                        tc_commit(&sh.u_full[i]);
+                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
+                        tc_commit(&sh.u_full[0]);
+                        tc_commit(&sh.u_full[1]);
                         TLW_END(6);
                     }
                     tc_commit(&sh.empty[s]);
