@@ -34,10 +34,16 @@ constexpr int D = 128;                // head size
 constexpr int WARP_TMA = 0, WARP_MMA = 1, TILE_W0 = 2, STATE_W0 = 10;
 constexpr int GATE_W0 = 18;               // warps 18,19: gates, decay mask M, per-token factors
 constexpr int NTHREADS = 20 * 32;
-constexpr int STAGE_BYTES = 5 * 16384;   // [K/K~1][K~2][Q/Q~1][Q~2][V]
-constexpr int OFF_K = 0, OFF_Q = 32768, OFF_V = 65536;
-constexpr int OFF_PT = 2 * STAGE_BYTES;  // P~ double buffer, 8 KB each
-constexpr int OFF_MASK = OFF_PT + 2 * 8192;  // decay mask M, bf16 [2][64][MASK_PITCH] (one buffer per chunk parity)
+// Shared-memory tiles (16 KB each, 128-byte swizzle).  K and Q land in one of three buffers and are scaled in
+// place for state 1; the state-2 copies and V live in one of two buffers.  The third landing buffer takes the TMA
+// latency and the score MMAs off the chain "operands of chunk c -> MMAs of chunk c -> buffers free again".
+constexpr int KQ_BYTES = 2 * 16384;      // [K / K~1][Q / Q~1]
+constexpr int KQ_Q = 16384;
+constexpr int X_BYTES = 3 * 16384;       // [K~2][Q~2][V]
+constexpr int X_Q = 16384, X_V = 32768;
+constexpr int OFF_X = 3 * KQ_BYTES;
+constexpr int OFF_PT = OFF_X + 2 * X_BYTES;  // P~, 8 KB (freed as soon as the V part of the output has read it)
+constexpr int OFF_MASK = OFF_PT + 8192;      // decay mask M, bf16 [2][64][MASK_PITCH] (one buffer per chunk parity)
 constexpr int MASK_PITCH = 72;               // bf16 elements; 144-byte rows keep 16-byte row accesses conflict-free
 constexpr int MASK_BYTES = 64 * MASK_PITCH * 2;
 constexpr int SMEM_TILES = OFF_MASK + 2 * MASK_BYTES;
@@ -104,7 +110,9 @@ struct alignas(16) GateSmem {
 };
 
 struct alignas(16) Shared {
-    uint64_t full[4], empty[4], p_full[2], p_free, prep_ready[2], sb_ready[2], s_ready[2], o_full[2], o_free, u_full[2], m_ready[2], m_free[2];
+    uint64_t kq_full[3], kq_empty[3], v_full[2], x_empty[2], p_full[2], p_free, pt_free, prep_ready[2], sb_ready[2], s_ready[2], o_full[2], o_free,
+        u_full[2], m_ready[2], m_free[2];
+    uint64_t full[4], empty[4];   // summary kernel
     uint32_t tmem_base;
     int abort_flag;
     GateSmem gs[2];
@@ -235,8 +243,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #endif
 
     if (tid == 0) {
-        mbar_init(&sh.full[0], 1); mbar_init(&sh.full[1], 1);
-        mbar_init(&sh.empty[0], 2); mbar_init(&sh.empty[1], 2);   // both issuers release a stage
+        for (int i = 0; i < 3; ++i) { mbar_init(&sh.kq_full[i], 1); mbar_init(&sh.kq_empty[i], 2); }   // both issuers release a buffer
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh.v_full[i], 1); mbar_init(&sh.x_empty[i], 2); }
+        mbar_init(&sh.pt_free, 1);
         mbar_init(&sh.p_full[0], 1); mbar_init(&sh.p_free, 8);   // every tile warp passes p_full before P is overwritten
         mbar_init(&sh.prep_ready[0], 8);
         mbar_init(&sh.sb_ready[0], 4); mbar_init(&sh.sb_ready[1], 4); mbar_init(&sh.s_ready[0], 4); mbar_init(&sh.s_ready[1], 4);
@@ -255,30 +264,68 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
     if (warp == WARP_TMA) {
         // ------------------------------------------------------------------ TMA producer + issuer of P and the state updates
-        // Two threads issue the MMAs of a chunk.  This one loads the tiles, issues the scores P = Q K^T of the next
-        // chunk as soon as its tile has landed and P of this chunk has been read, and the state updates
-        // S^i^T += V^T K~i (which wait only for the state warps' rescale); the other issues everything that
-        // accumulates into the output tile.
+        // Two threads issue the MMAs of a chunk.  This one loads the tiles, issues the state updates
+        // S^i^T += V^T K~i (which wait only for the state warps' rescale) and the scores P = Q K^T two chunks ahead;
+        // the other issues everything that accumulates into the output tile.
         if (lane == 0) {
             prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);
-            constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
-            constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4);
-            const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dk0 = smem_desc_sw128(sa + OFF_K, 16, 1024);
-            const uint64_t dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024), dkn0 = smem_desc_sw128(sa + OFF_K, 8192, 1024);
-            // iterations -2 and -1 only start the first two loads and the first scores
+            constexpr uint32_t ID_U = idesc_bf16(128, 128, 1, 1);
+            constexpr uint64_t KQ_STEP = (uint64_t)(KQ_BYTES >> 4), X_STEP = (uint64_t)(X_BYTES >> 4);
+            const uint64_t dq0 = smem_desc_sw128(sa + KQ_Q, 16, 1024), dk0 = smem_desc_sw128(sa, 16, 1024);         // K-major (scores)
+            const uint64_t dkn1 = smem_desc_sw128(sa, 8192, 1024), dkn2 = smem_desc_sw128(sa + OFF_X, 8192, 1024);   // K~1, K~2 as N operands
+            const uint64_t dv0 = smem_desc_sw128(sa + OFF_X + X_V, 8192, 1024);
+            // Iteration c: state updates of chunk c, refills of the buffers chunk c used, scores of chunk c + 2.
+            // Iterations -3..-1 only start the first loads and the first two score tiles (one copy of each code path).
+            int k3 = 0, ph3 = 0;        // c mod 3 and the parity of c / 3 (valid for c >= 0)
+            int k3p = 0;                // (c + 2) mod 3 for c >= -2
 #pragma unroll 1
-            for (int c = -2; c < nc; ++c) {
+            for (int c = -3; c < nc; ++c) {
                 const int s = c & 1;
-                const uint64_t so = (uint64_t)s * STAGE_STEP;
-                if (c >= -1 && c + 1 < nc) {
-                    // P_{c+1}: K-major operands, four 32-byte k-steps inside a 64-element block, the next block 8 KB further
-                    WAITP(3, &sh.full[s ^ 1], ((c + 1) >> 1) & 1);
-                    if (c >= 0) WAITP(4, &sh.p_free, c & 1);            // every tile warp has seen P_c
-                    TL(4, c + 1, 1);
+                if (c >= 0) {
+                    WAITP(0, &sh.prep_ready[0], c & 1);            // K~1, K~2 are in place
+                    WAITP(3, &sh.v_full[s], (c >> 1) & 1);
+                    TL(4, c, 3);
+                    const uint64_t a = dv0 + (uint64_t)s * X_STEP;
+#pragma unroll 1
+                    for (int i = 0; i < 2; ++i) {
+                        WAITP(1, &sh.s_ready[i], c & 1);           // fp32 state i has been rescaled
+                        TL(4, c, 4 + i);
+                        tc_fence_after();
+                        const uint64_t b = i == 0 ? dkn1 + (uint64_t)k3 * KQ_STEP : dkn2 + (uint64_t)s * X_STEP;
+                        TLW_BEGIN;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S + 128 * i, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
+                        tc_commit(&sh.u_full[i]);
+                        TLW_END(6);
+                    }
+                    tc_commit(&sh.kq_empty[k3]);
+                    tc_commit(&sh.x_empty[s]);
+                    TL(4, c, 6);
+                }
+                if (c + 3 < nc) {
+                    if (c >= 0) WAITP(2, &sh.kq_empty[k3], ph3);   // both issuers' MMAs on this buffer are done
+                    if (c >= 0) TL(4, c, 7);
+                    const int i3 = c >= 0 ? k3 : c + 3;
+                    uint8_t* dst = tiles + i3 * KQ_BYTES;
+                    const int t = t0 + (c + 3) * C;
+                    mbar_arrive_expect_tx(&sh.kq_full[i3], 4 * 8192);
+                    tma_load_4d(dst, &map_k, &sh.kq_full[i3], 0, t, 0, h);
+                    tma_load_4d(dst + KQ_Q, &map_q, &sh.kq_full[i3], 0, t, 0, h);
+                    TL(4, c + 3, 0);
+                }
+                if (c >= -2 && c + 2 < nc) {
+                    if (c >= 0) WAITP(2, &sh.x_empty[s], (c >> 1) & 1);
+                    mbar_arrive_expect_tx(&sh.v_full[s], 2 * 8192);
+                    tma_load_4d(tiles + OFF_X + s * X_BYTES + X_V, &map_v, &sh.v_full[s], 0, t0 + (c + 2) * C, 0, h);
+                    // scores of chunk c + 2: K-major operands, four 32-byte k-steps inside a 64-element block, the next block 8 KB further
+                    const int cp = c + 2;
+                    WAITP(4, &sh.kq_full[k3p], (cp / 3) & 1);
+                    if (cp >= 1) WAITP(4, &sh.p_free, (cp - 1) & 1);          // every tile warp has seen the previous P
+                    TL(4, cp, 1);
                     tc_fence_after();
-                    const uint64_t sn = (uint64_t)(s ^ 1) * STAGE_STEP;
+                    const uint64_t sn = (uint64_t)k3p * KQ_STEP;
                     TLW_BEGIN;
 #pragma unroll 1
                     for (int blk = 0; blk < 2; ++blk) {
@@ -288,46 +335,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     }
                     tc_commit(&sh.p_full[0]);
                     TLW_END(5);
-                    TL(4, c + 1, 2);
+                    TL(4, cp, 2);
                 }
-                if (c >= 0) {
-                    WAITP(0, &sh.prep_ready[0], c & 1);     // K~1, K~2 are in the stage
-                    TL(4, c, 3);
-                    // both states in one N = 256 MMA per k-step: [S1^T S2^T] += V^T [K~1 K~2] (the two K~ tiles and the two
-                    // fp32 states are adjacent), so V^T is read from shared memory once
-                    WAITP(1, &sh.s_ready[0], c & 1);        // fp32 states have been rescaled
-                    WAITP(1, &sh.s_ready[1], c & 1);
-                    TL(4, c, 5);
-                    tc_fence_after();
-                    {
-                        const uint64_t a = dv0 + so, b = dkn0 + so;
-                        TLW_BEGIN;
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_S, a + (uint64_t)(kk * 128), b + (uint64_t)(kk * 128), ID_U, 1);
-                        tc_commit(&sh.u_full[0]);
-                        tc_commit(&sh.u_full[1]);
-                        TLW_END(6);
-                    }
-                    tc_commit(&sh.empty[s]);
-                    TL(4, c, 6);
-                }
-                if (c + 2 < nc) {
-                    if (c >= 0) WAITP(2, &sh.empty[s], (c >> 1) & 1);   // both issuers' MMAs on this stage are done
-                    if (c >= 0) TL(4, c, 7);
-                    TLW_BEGIN;
-                    uint8_t* st = tiles + s * STAGE_BYTES;
-                    const int t = t0 + (c + 2) * C;
-                    mbar_arrive_expect_tx(&sh.full[s], 6 * 8192);
-                    tma_load_4d(st + OFF_Q, &map_q, &sh.full[s], 0, t, 0, h);
-                    tma_load_4d(st + OFF_K, &map_k, &sh.full[s], 0, t, 0, h);
-                    tma_load_4d(st + OFF_V, &map_v, &sh.full[s], 0, t, 0, h);
-                    if (c + 4 < nc) {   // pull the tile after next into L2 while this one is in flight
-                        const int t2 = t + 2 * C;
-                        tma_prefetch_4d(&map_q, 0, t2, 0, h); tma_prefetch_4d(&map_k, 0, t2, 0, h); tma_prefetch_4d(&map_v, 0, t2, 0, h);
-                    }
-                    TLW_END(7);
-                    TL(4, c + 2, 0);
-                }
+                if (c >= 0 && ++k3 == 3) { k3 = 0; ph3 ^= 1; }
+                if (c >= -2 && ++k3p == 3) k3p = 0;
             }
             TL_DUMP(0);
         }
@@ -340,23 +351,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_OS = idesc_bf16(128, 64, 0, 0);
             constexpr uint32_t ID_OV = idesc_bf16(128, 64, 1, 0);
-            constexpr uint64_t STAGE_STEP = (uint64_t)(STAGE_BYTES >> 4), PT_STEP = (uint64_t)(8192 >> 4);
-            const uint64_t dq0 = smem_desc_sw128(sa + OFF_Q, 16, 1024), dv0 = smem_desc_sw128(sa + OFF_V, 8192, 1024);
+            constexpr uint64_t KQ_STEP = (uint64_t)(KQ_BYTES >> 4), X_STEP = (uint64_t)(X_BYTES >> 4);
+            const uint64_t dq1 = smem_desc_sw128(sa + KQ_Q, 16, 1024), dq2 = smem_desc_sw128(sa + OFF_X + X_Q, 16, 1024);
+            const uint64_t dv0 = smem_desc_sw128(sa + OFF_X + X_V, 8192, 1024);
             const uint64_t dp0 = smem_desc_sw128(sa + OFF_PT, 16, 1024);
+            int k3 = 0;
 #pragma unroll 1
             for (int c = 0; c < nc; ++c) {
                 const int s = c & 1;
-                const uint64_t so = (uint64_t)s * STAGE_STEP;
                 TL(1, c, 0);
                 WAITP(0, &sh.prep_ready[0], c & 1);
+                WAITP(3, &sh.v_full[s], (c >> 1) & 1);
                 if (c > 0) WAITP(1, &sh.o_free, (c - 1) & 1);
                 TL(1, c, 1);
                 tc_fence_after();
                 {
                     TLW_BEGIN;
-                    const uint64_t a = dv0 + so, b = dp0 + (uint64_t)s * PT_STEP;
+                    const uint64_t a = dv0 + (uint64_t)s * X_STEP;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, a + (uint64_t)(kk * 128), b + (uint64_t)(2 * kk), ID_OV, kk ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_O, a + (uint64_t)(kk * 128), dp0 + (uint64_t)(2 * kk), ID_OV, kk ? 1u : 0u);
+                    tc_commit(&sh.pt_free);       // P~ may be overwritten
                     TLW_END(4);
                     TL(1, c, 2);
                 }
@@ -366,7 +380,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     TL(1, c, 3 + i);
                     tc_fence_after();
                     TLW_BEGIN;
-                    const uint64_t dq = dq0 + so + (uint64_t)(i * (16384 >> 4));
+                    const uint64_t dq = i == 0 ? dq1 + (uint64_t)k3 * KQ_STEP : dq2 + (uint64_t)s * X_STEP;
                     const uint32_t at = tb + COL_SB + 64 * i;
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_O, at + 8 * kk, dq + (uint64_t)(2 * kk), ID_OS, 1);
@@ -375,73 +389,36 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     TLW_END(5);
                 }
                 tc_commit(&sh.o_full[0]);
-                tc_commit(&sh.empty[s]);
+                tc_commit(&sh.kq_empty[k3]);
+                tc_commit(&sh.x_empty[s]);
                 TL(1, c, 6);
+                if (++k3 == 3) k3 = 0;
             }
             TL_DUMP(1);
         }
     } else if (warp < STATE_W0) {
         // ------------------------------------------------------------------ tile warps 2..9
-        // All eight warps work on every chunk: P~ = P (.) M (the four warps of quadrants 0 and 1), the scaled
-        // copies of Q and K (everyone), and the outputs of the previous chunk (everyone: lanes = d_v).
+        // All eight warps work on every chunk: P~ = P (.) M (the four warps of quadrants 0 and 1) and the scaled
+        // copies of Q and K (everyone).
         const int tt = tid - TILE_W0 * 32;                // 0..255
         const int q = warp & 3;                           // TMEM lane quadrant
         const int half = (warp - TILE_W0) >> 2;           // column half: 32 score columns / 32 output tokens
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
-        __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
 
-        // chunk c: each thread owns one d_v lane of O^T and 32 tokens; a warp's store of one token is 64 contiguous
-        // bytes (two full sectors), so the outputs go straight from registers to global memory
-        auto outputs = [&](int c) {
-            WAITP(0, &sh.o_full[0], c & 1);
-            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 3);
-            tc_fence_after();
-            TLT(tlo0);
-            uint32_t r[32];
-            tmem_ld32(lane_addr + COL_O + 32 * half, r);
-            tc_wait_ld();
-            TLT(tlo1); TLACC(5, tlo1 - tlo0);
-            __syncwarp();
-            if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
-            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 4);
-            const int valid = min(C, sq.len - tok0 - c * C) - 32 * half;     // tokens of this warp's half that exist
-            __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * half) * p.H + h) * D + 32 * q + lane;
-            const size_t row = (size_t)p.H * D;
-            if (valid >= 32) {
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) dst[jj * row] = __float2bfloat16_rn(__uint_as_float(r[jj]));
-            } else {
-#pragma unroll 1
-                for (int jj = 0; jj < valid; ++jj) {   // ragged tail (cold): pick the register with a shuffle-free select chain
-                    float x = 0.f;
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) x = e == jj ? __uint_as_float(r[e]) : x;
-                    dst[jj * row] = __float2bfloat16_rn(x);
-                }
-            }
-            TLACC(6, clock64() - tlo1);
-            if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 5);
-        };
-
-        // Iteration c builds the operands of chunk c (c < nc) and stores the outputs of chunk c-1 (c > 0); the
-        // outputs go first when they are already there, otherwise after the operands.  One code copy of each.
-        for (int c = 0; c <= nc; ++c) {
+        int k3 = 0, ph3 = 0;      // c mod 3, parity of c / 3
+        for (int c = 0; c < nc; ++c, k3 = k3 == 2 ? 0 : k3 + 1, ph3 ^= (k3 == 0)) {
             const int s = c & 1;
             GateSmem& gs = sh.gs[s];
-            uint8_t* st = tiles + s * STAGE_BYTES;
+            uint8_t* kq = tiles + k3 * KQ_BYTES;            // K (-> K~1) and Q (-> Q~1) of this chunk
+            uint8_t* xb = tiles + OFF_X + s * X_BYTES;      // K~2, Q~2 (and V) of this chunk
             const uint8_t* Mm = tiles + OFF_MASK + s * MASK_BYTES;
             if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 0);
-            bool out_done = c == 0;
-#pragma unroll 1
-            for (int pass = 0; pass < 2; ++pass) {
-                if (!out_done && (pass == 1 || c == nc || mbar_test_wait(&sh.o_full[0], (c - 1) & 1))) {
-                    outputs(c - 1);
-                    out_done = true;
-                }
-                if (pass == 1 || c == nc) continue;
+            {
                 WAITP(2, &sh.m_ready[s], (c >> 1) & 1);
-                WAITP(3, &sh.full[s], (c >> 1) & 1);
-                WAITP(4, &sh.p_full[0], c & 1);   // P ready; the MMA is also done reading raw Q, K
+                WAITP(3, &sh.kq_full[k3], ph3);   // TMA writes of K, Q visible to this thread
+                // P ready: the MMA is done reading raw Q, K.  The second issuer put P_c behind its wait for the MMAs of
+                // chunk c - 2, so the K~2 / Q~2 buffer of this parity is free as well.
+                WAITP(4, &sh.p_full[0], c & 1);
                 tc_fence_after();
                 if ((warp == 4 || warp == 6) && lane == 0) TL(warp == 4 ? 2 : 5, c, 1);
                 TLT(tlm0);
@@ -449,12 +426,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (q < 2) {
                     // ---- P~ rows 32q..32q+31, columns 32 half .. +31
                     const int j = 32 * q + lane;
-                    uint8_t* pt = tiles + OFF_PT + s * 8192;
+                    uint8_t* pt = tiles + OFF_PT;
                     const bool any = half <= q;               // block not entirely above the diagonal
                     uint32_t r[32];
                     if (any) { tmem_ld32(lane_addr + COL_P + 32 * half, r); tc_wait_ld(); }
                     __syncwarp();
                     if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
+                    if (c >= 1) WAITP(1, &sh.pt_free, (c - 1) & 1);     // the V part of chunk c - 1 has read P~
                     const uint4* mrow = reinterpret_cast<const uint4*>(Mm + j * (MASK_PITCH * 2) + 64 * half);
 #pragma unroll
                     for (int m4 = 0; m4 < 4; ++m4) {
@@ -480,14 +458,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int m = 0; m < 4; ++m) {
                         const int idx = tt + 256 * m;             // 16-byte piece inside a 16 KB tile
                         const int row = (idx >> 3) & 63;
-                        uint4* qp = reinterpret_cast<uint4*>(st + OFF_Q) + idx;
-                        uint4* kp = reinterpret_cast<uint4*>(st + OFF_K) + idx;
-                        const uint4 xq = *qp, xk = *kp;
+                        const uint4 xq = reinterpret_cast<const uint4*>(kq + KQ_Q)[idx], xk = reinterpret_cast<const uint4*>(kq)[idx];
                         const uint32_t f0 = gs.rowf[0][row], f1 = gs.rowf[1][row], w0 = gs.w[0][row], w1 = gs.w[1][row];
-                        *qp = scale8(xq, f0);
-                        *(qp + 1024) = scale8(xq, f1);
-                        *kp = scale8(xk, w0);
-                        *(kp + 1024) = scale8(xk, w1);
+                        reinterpret_cast<uint4*>(kq + KQ_Q)[idx] = scale8(xq, f0);
+                        reinterpret_cast<uint4*>(xb + X_Q)[idx] = scale8(xq, f1);
+                        reinterpret_cast<uint4*>(kq)[idx] = scale8(xk, w0);
+                        reinterpret_cast<uint4*>(xb)[idx] = scale8(xk, w1);
                     }
                 }
                 TLACC(9, clock64() - tlm1);
@@ -584,6 +560,33 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const uint32_t sb_addr = lane_addr + COL_SB + 64 * hi;
         const int v = 32 * q + lane;
         const float* gsrc = hi == 0 ? p.g_hist : p.g_rec;
+        // Outputs of chunk c, tokens 32 hi .. 32 hi + 31 of this warp's lane quadrant: each thread owns one d_v lane of
+        // O^T; a warp's store of one token is 64 contiguous bytes (two full sectors), so the values go straight from
+        // registers to global memory.  The state warps do this after their pass over the state, in the time they would
+        // otherwise wait for the next update MMA.
+        __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
+        auto outputs = [&](int c) {
+            uint32_t r[32];
+            tmem_ld32(lane_addr + COL_O + 32 * hi, r);
+            tc_wait_ld();
+            __syncwarp();
+            if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.o_free); }
+            const int valid = min(C, sq.len - tok0 - c * C) - 32 * hi;     // tokens of this warp's half that exist
+            __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * hi) * p.H + h) * D + v;
+            const size_t row = (size_t)p.H * D;
+            if (valid >= 32) {
+#pragma unroll
+                for (int jj = 0; jj < 32; ++jj) dst[jj * row] = __float2bfloat16_rn(__uint_as_float(r[jj]));
+            } else {
+#pragma unroll 1
+                for (int jj = 0; jj < valid; ++jj) {   // ragged tail (cold): pick the register with a shuffle-free select chain
+                    float x = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x = e == jj ? __uint_as_float(r[e]) : x;
+                    dst[jj * row] = __float2bfloat16_rn(x);
+                }
+            }
+        };
         // chunk decay a = prod of this state's gates over the chunk (two tokens per lane).  The gates of chunk c + 1
         // are requested at the top of iteration c and multiplied together at its end, so the load latency hides
         // behind the waits and the two passes.
@@ -662,6 +665,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (warp == 12 && lane == 0) TL(3, c, 2);
             if (warp == 16 && lane == 0) TL(3, c, 5);
             TLT(tls1); TLACC(2, tls1 - tls0);
+            outputs(c - 1);       // o_full of chunk c - 1 was awaited at the top of this iteration
             TLACC(3, clock64() - tls1);
             a_next = warp_prod(gp_next);
             if (warp == 12 && lane == 0) TL(3, c, 3);
@@ -669,7 +673,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         if (warp == 12 && lane == 0) TL_DUMP(4);
         if (warp == 16 && lane == 0) TL_DUMP(5);
-        // ---- final states of this segment's last chunk
+        // ---- outputs of the last chunk, final states of this segment
+        mbar_wait(&sh.o_full[0], (nc - 1) & 1, abortp, p.status);
+        tc_fence_after();
+        outputs(nc - 1);
         mbar_wait(&sh.u_full[hi], (nc - 1) & 1, abortp, p.status);
 #ifdef DSLA_TIMELINE
         if (warp == 12 && lane == 0 && g_timeline) g_timeline[3072 + 4 * blockIdx.x + 3] = gtime();
