@@ -51,6 +51,8 @@ constexpr int SMEM_DYN = SMEM_TILES + 1024;  // + alignment slack
 // summary kernel: 4 stages of [K/K~1][K~2][V]
 constexpr int SUM_STAGES = 4, SUM_STAGE_BYTES = 3 * 16384, SUM_OFF_V = 32768;
 constexpr int SUM_NTHREADS = 384, SUM_NCOMPUTE = 256;
+constexpr int SUM_GATE_AHEAD = 6;        // chunks between the L2 prefetch and the load of a chunk's gates
+constexpr int SUM_PREFETCH = 8;          // chunks between the L2 prefetch and the load of a tile
 constexpr int SUM_SMEM_DYN = SUM_STAGES * SUM_STAGE_BYTES + 1024;
 // TMEM columns
 constexpr uint32_t COL_S = 0;      // fp32 S1^T [0,128), S2^T [128,256)
@@ -74,7 +76,11 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 #define TLW_END(tag) tl_w[tag] += clock64() - _tlb
 #define TL_DUMP(role) do { if (tlp) { for (int _k = 0; _k < 10; ++_k) tlp[3800 + 12 * (role) + _k] = tl_w[_k]; tlp[3800 + 12 * (role) + 10] = clock64() - tl_t0; } } while (0)
 #else
+#ifdef DSLA_TIMELINE_SUMMARY   // events of the summary kernel only
+#define TL_INIT long long* const tlp = nullptr
+#else
 #define TL_INIT long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr
+#endif
 #define WAITP(tag, bar, ph) mbar_wait(bar, ph, abortp, p.status)
 #define TLT(var) do { } while (0)
 #define TLACC(tag, expr) do { } while (0)
@@ -714,6 +720,11 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     if (threadIdx.x == 0 && g_timeline) g_timeline[4096 + 4 * blockIdx.x] = gtime();
 #endif
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main grid may be scheduled as SMs become free
+#ifdef DSLA_TIMELINE_SUMMARY
+    long long* const tlp = (int)blockIdx.x == g_timeline_block ? g_timeline : nullptr;
+#else
+    long long* const tlp = nullptr; (void)tlp;
+#endif
     const int nsum = tp.nseg - 1;
     const int g = blockIdx.x % nsum;
     const int h = (blockIdx.x / nsum) % p.H;
@@ -748,12 +759,19 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
             for (int it = 0; it < nc; ++it) {
                 const int s = it % SUM_STAGES, u = it / SUM_STAGES;
+                TL(0, it, 0);
                 if (u >= 1) mbar_wait(&sh.empty[s], (u - 1) & 1, abortp, p.status);
+                TL(0, it, 1);
                 uint8_t* st = tiles + s * SUM_STAGE_BYTES;
                 const int t = t0 + (nc - 1 - it) * C;
                 mbar_arrive_expect_tx(&sh.full[s], 4 * 8192);
                 tma_load_4d(st, &map_k, &sh.full[s], 0, t, 0, h);
                 tma_load_4d(st + SUM_OFF_V, &map_v, &sh.full[s], 0, t, 0, h);
+                if (it + SUM_PREFETCH < nc) {   // pull a tile well ahead into L2: the four stages alone do not cover the HBM latency
+                    const int tp2 = t - SUM_PREFETCH * C;
+                    tma_prefetch_4d(&map_k, 0, tp2, 0, h);
+                    tma_prefetch_4d(&map_v, 0, tp2, 0, h);
+                }
             }
         }
     } else if (warp == 9) {
@@ -762,41 +780,55 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
             for (int it = 0; it < nc; ++it) {
                 const int s = it % SUM_STAGES, u = it / SUM_STAGES;
+                TL(1, it, 0);
                 mbar_wait(&k_ready[s], u & 1, abortp, p.status);
+                TL(1, it, 1);
                 tc_fence_after();
                 const uint32_t st = sa + s * SUM_STAGE_BYTES;
                 const uint64_t dv = smem_desc_sw128(st + SUM_OFF_V, 8192, 1024), dkk = smem_desc_sw128(st, 8192, 1024);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) mma_ss(tb, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, (it | kk) > 0);
                 tc_commit(&sh.empty[s]);
+                TL(1, it, 2);
                 if (it == nc - 1) tc_commit(&sh.u_full[0]);
             }
         }
     } else if (warp >= 10) {
-        // ---- weights: warp 10 the history state, warp 11 the recency state; lane l holds tokens l and l + 32
+        // ---- weights: warp 10 the history state, warp 11 the recency state; lane l holds the adjacent tokens 2l and 2l + 1,
+        // so one suffix scan over the 32 pair products gives every token's weight
         const int i = warp - 10;
         const float* gsrc = i == 0 ? p.g_hist : p.g_rec;
         float R = 1.f;                                 // product of the gates of all later chunks
-        float nl = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + lane, p.H, h, true), 0.f);
-        float nh = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + lane + 32, p.H, h, true), 0.f);
+        float n0 = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane, p.H, h, true), 0.f);
+        float n1 = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane + 1, p.H, h, true), 0.f);
         for (int it = 0; it < nc; ++it) {
             const int s = it % SUM_STAGES, u = it / SUM_STAGES;
-            const float xl = nl, xh = nh;
+            const float g0 = n0, g1 = n1;
             if (it + 1 < nc) {
-                const int t = t0 + (nc - 2 - it) * C + lane;
-                nl = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
-                nh = fmaxf(load_gate(gsrc, t + 32, p.H, h, true), 0.f);
+                const int t = t0 + (nc - 2 - it) * C + 2 * lane;
+                n0 = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
+                n1 = fmaxf(load_gate(gsrc, t + 1, p.H, h, true), 0.f);
             }
-            const float sh_in = warp_suffix_prod(xh, lane), sl_in = warp_suffix_prod(xl, lane);
-            const float tot_hi = __shfl_sync(0xffffffffu, sh_in, 0), tot_lo = __shfl_sync(0xffffffffu, sl_in, 0);
-            float sh_ex = __shfl_down_sync(0xffffffffu, sh_in, 1), sl_ex = __shfl_down_sync(0xffffffffu, sl_in, 1);
-            if (lane == 31) { sh_ex = 1.f; sl_ex = 1.f; }
+            if (it + 1 + SUM_GATE_AHEAD < nc) {
+                // One chunk of look-ahead does not cover the DRAM latency (this warp's iteration is shorter): pull the gates
+                // of a chunk further ahead into L2 so that the load above becomes an L2 hit.
+                const float* gp = gsrc + (size_t)(t0 + (nc - 2 - it - SUM_GATE_AHEAD) * C + 2 * lane) * p.H + h;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(gp));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(gp + p.H));
+            }
+            const float sfx = warp_suffix_prod(g0 * g1, lane);        // product of the gates of tokens >= 2l
+            const float tot = __shfl_sync(0xffffffffu, sfx, 0);
+            float ex = __shfl_down_sync(0xffffffffu, sfx, 1);         // ... of tokens > 2l + 1
+            if (lane == 31) ex = 1.f;
+            ex *= R;
+            if (warp == 10 && lane == 0) TL(3, it, 0);
             if (u >= 1) mbar_wait(&w_free[s], (u - 1) & 1, abortp, p.status);
-            wts[s][i][lane] = dup_bf16(sl_ex * tot_hi * R);
-            wts[s][i][lane + 32] = dup_bf16(sh_ex * R);
-            R *= tot_lo * tot_hi;
+            if (warp == 10 && lane == 0) TL(3, it, 1);
+            *reinterpret_cast<uint2*>(&wts[s][i][2 * lane]) = make_uint2(dup_bf16(g1 * ex), dup_bf16(ex));
+            R *= tot;
             __syncwarp();
             if (lane == 0) mbar_arrive(&w_ready[s]);
+            if (warp == 10 && lane == 0) TL(3, it, 2);
         }
         if (lane == 0) out[2 * D * D + i] = R;         // A_g: product of every gate of the segment
     } else {
@@ -806,12 +838,15 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
         for (int it = 0; it < nc; ++it) {
             const int s = it % SUM_STAGES, u = it / SUM_STAGES;
             uint8_t* st = tiles + s * SUM_STAGE_BYTES;
+            if (tid == 0) TL(2, it, 0);
             mbar_wait(&w_ready[s], u & 1, abortp, p.status);
+            if (tid == 0) TL(2, it, 1);
             mbar_wait(&sh.full[s], u & 1, abortp, p.status);
+            if (tid == 0) TL(2, it, 2);
 #ifdef DSLA_TIMELINE
             if (tid == 0 && it == 0 && g_timeline) g_timeline[4096 + 4 * blockIdx.x + 2] = gtime();
 #endif
-#pragma unroll 2
+#pragma unroll
             for (int m = 0; m < 4; ++m) {
                 const int idx = tid + SUM_NCOMPUTE * m;
                 const int row = (idx >> 3) & 63;
@@ -824,6 +859,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) { mbar_arrive(&k_ready[s]); mbar_arrive(&w_free[s]); }
+            if (tid == 0) TL(2, it, 3);
         }
         mbar_wait(&sh.u_full[0], 0, abortp, p.status);
 #ifdef DSLA_TIMELINE
