@@ -29,6 +29,31 @@ def test_tensor_prefill_ragged_slots_initial_state():
     check_prefill(inp, state0=st0, slots=slots, num_slots=8, impl="tensor", scale=0.5)
 
 
+def test_tensor_prefill_packed_batch_longest_first():
+    """More (sequence, head) pairs than SMs: no split, blocks visit the sequences by descending length (ties,
+    empty sequences and a ragged last chunk included); slots are permuted so a wrong sequence index shows."""
+    rng = np.random.default_rng(8600)
+    lens = [int(x) for x in rng.integers(1, 400, size=38)] + [0, 257, 257, 64]
+    inp = gen.make_packed(8601, lens, 4, 128, BF)
+    slots = [int(x) for x in rng.permutation(len(lens))]
+    check_prefill(inp, slots=slots, num_slots=len(lens), impl="tensor")
+
+
+def test_tensor_prefill_ragged_batch_split_into_segments():
+    """Few pairs with very different lengths: every sequence is cut with the longest one's segment plan, so short
+    sequences leave later segments empty; summaries, their fold into the initial state and the order array all run."""
+    inp = gen.make_packed(8700, [3000, 700, 65, 0, 1], 2, 128, BF)
+    check_prefill(inp, impl="tensor")
+    st0 = gen.make_states(8701, 5, 2, 128, 128, std=0.3).numpy()
+    check_prefill(inp, state0=st0, impl="tensor")
+
+
+@pytest.mark.parametrize("T", [64 * 40, 64 * 200 + 17])
+def test_tensor_prefill_single_head_sixteen_segments(T):
+    """One (sequence, head) pair: the deepest split (up to 16 segments, later ones shorter than earlier ones)."""
+    check_prefill(gen.make_dense(8800 + T % 97, 1, T, 1, 128, BF), impl="tensor")
+
+
 @pytest.mark.parametrize("pattern", ["ones", "zeros", "single_zero", "alternating", "swapped", "tiny"])
 def test_tensor_prefill_gate_patterns(pattern):
     T, H, d = 600, 2, 128
