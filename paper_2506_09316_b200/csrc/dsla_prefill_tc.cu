@@ -8,13 +8,15 @@
 //     S^i^T <- a^i S^i^T + V^T (w^i (.) K)                            rescale on CUDA cores, MMA accumulates
 // Everything is computed transposed (d_v on the 128 TMEM lanes, tokens or d_k on the columns) so
 // every MMA has M = 128.  The two fp32 states live in TMEM for the whole sequence; a bf16 copy in
-// TMEM is the A operand of the readout.  TMA stages Q/K/V tiles (128-byte swizzle, 2 stages).
+// TMEM is the A operand of the readout.  TMA lands K and Q in one of three buffers and V in one of
+// two (128-byte swizzle); the gate terms come from cumulative log2-gates of the chunk.
 //
 // A sequence may be split into `nseg` segments along T so that few (sequence, head) pairs still
 // fill the GPU: a first kernel computes each segment's state summary from zero
 // (U_g = sum_s (prod of later gates in the segment) k_s^T v_s and A_g = prod of the segment's
-// gates) into the workspace; the main kernel combines the summaries of earlier segments into its
-// initial state and then runs its segment.
+// gates) into the workspace; the main kernel, launched as its programmatic dependent, combines the
+// summaries of earlier segments into its initial state and then runs its segment.  Packed batches
+// are visited longest sequence first.
 #include <type_traits>
 
 #include "dsla_internal.cuh"
@@ -28,8 +30,9 @@ namespace {
 
 constexpr int C = 64;                 // tokens per chunk
 constexpr int D = 128;                // head size
-// Warp roles of the main kernel: 0 = TMA producer, 1 = MMA issuer, 2..9 = tile warps (gates, decay mask,
-// operand scaling), 10..17 = state warps (state rescale + bf16 copy, outputs, initial/final state).
+// Warp roles of the main kernel: 0 = TMA producer that also issues the score and state-update MMAs, 1 = issuer of
+// the MMAs that build the output tile, 2..9 = tile warps (masked scores, operand scaling), 10..17 = state warps
+// (state rescale + bf16 copy, outputs, initial/final state), 18..19 = gate warps.
 // A warp may touch only the 32 TMEM lanes of its quadrant (warp index mod 4).
 constexpr int WARP_TMA = 0, WARP_MMA = 1, TILE_W0 = 2, STATE_W0 = 10;
 constexpr int GATE_W0 = 18;               // warps 18,19: gates, decay mask M, per-token factors
