@@ -17,8 +17,6 @@
 // gates) into the workspace; the main kernel, launched as its programmatic dependent, combines the
 // summaries of earlier segments into its initial state and then runs its segment.  Packed batches
 // are visited longest sequence first.
-#include <type_traits>
-
 #include "dsla_internal.cuh"
 #include "tc_utils.cuh"
 
