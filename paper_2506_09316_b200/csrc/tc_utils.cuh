@@ -32,9 +32,9 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait.  The fast path (phase already complete) is a single inlined try_wait; otherwise a
-// non-inlined loop polls.  It gives up after `limit` polls (each poll may itself suspend for a short,
-// hardware-chosen time), raises *abort_flag (shared) and *status (global) and returns false.  Once the
+// Bounded wait.  The fast path (phase already complete) is a single inlined test; otherwise a
+// non-inlined loop polls with a short sleep between tests.  It gives up after `limit` polls, raises
+// *abort_flag (shared) and *status (global) and returns false.  Once the
 // abort flag is up every later wait returns at once, so a CTA that lost a signal still runs to
 // its end, frees its TMEM and exits instead of hanging.
 __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
