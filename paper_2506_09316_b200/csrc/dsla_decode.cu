@@ -21,6 +21,11 @@ __global__ void __launch_bounds__(128) decode_kernel(const DecodeParams p) {
     const int r0 = tid >> 3;  // 0..15
     const int col = slab * 32 + c4 * 4;
 
+    // The kernel is launched as a programmatic dependent of whatever precedes it in the stream: it may become
+    // resident while that grid drains (hiding the launch latency), reads or writes nothing before this wait, and
+    // lets its own successor do the same.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int slot = p.slots ? p.slots[b] : b;
     T* o = reinterpret_cast<T*>(p.o) + ((size_t)b * p.H + h) * D;
     if (slot < 0 || slot >= p.num_slots) {
@@ -94,12 +99,23 @@ dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStrea
     if (p.B == 0) return DSLA_OK;
     const long long blocks = (long long)p.B * p.H * (d / 32);
     if (blocks > 0x7fffffffLL) return DSLA_ERR_UNSUPPORTED;
-    const dim3 grid((unsigned)blocks), block(128);
-    if (d == 128 && dt == DSLA_BF16) decode_kernel<128, __nv_bfloat16><<<grid, block, 0, s>>>(p);
-    else if (d == 128 && dt == DSLA_F32) decode_kernel<128, float><<<grid, block, 0, s>>>(p);
-    else if (d == 64 && dt == DSLA_BF16) decode_kernel<64, __nv_bfloat16><<<grid, block, 0, s>>>(p);
-    else if (d == 64 && dt == DSLA_F32) decode_kernel<64, float><<<grid, block, 0, s>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t rc;
+    if (d == 128 && dt == DSLA_BF16) rc = cudaLaunchKernelEx(&cfg, decode_kernel<128, __nv_bfloat16>, p);
+    else if (d == 128 && dt == DSLA_F32) rc = cudaLaunchKernelEx(&cfg, decode_kernel<128, float>, p);
+    else if (d == 64 && dt == DSLA_BF16) rc = cudaLaunchKernelEx(&cfg, decode_kernel<64, __nv_bfloat16>, p);
+    else if (d == 64 && dt == DSLA_F32) rc = cudaLaunchKernelEx(&cfg, decode_kernel<64, float>, p);
     else return DSLA_ERR_UNSUPPORTED;
+    if (rc != cudaSuccess) return DSLA_ERR_CUDA;
     count_launch();
     return cudaGetLastError() == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
 }

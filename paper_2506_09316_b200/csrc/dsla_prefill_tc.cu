@@ -243,6 +243,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int nc = sq.c_end - sq.c_begin;
     const int t0 = sq.t_begin + sq.c_begin * C;   // first token of this segment
     const int tok0 = sq.c_begin * C;              // its index inside the sequence
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch behind this grid (the decode step) may be scheduled early
     TL_INIT;
     if (tid == 0) TL(0, 63, 6);
 #ifdef DSLA_TIMELINE
