@@ -118,7 +118,7 @@ struct alignas(16) GateSmem {
 
 struct alignas(16) Shared {
     uint64_t kq_full[3], kq_empty[3], v_full[2], x_empty[2], p_full[2], p_free, pt_free, prep_ready[2], sb_ready[2], s_ready[2], o_full[2], o_free,
-        u_full[2], m_ready[2], m_free[2];
+        u_full[2], m_ready[2], m_free[2], init_done;
     uint64_t full[4], empty[4];   // summary kernel
     uint32_t tmem_base;
     int abort_flag;
@@ -174,11 +174,14 @@ __device__ __forceinline__ SeqInfo seq_info(const PrefillParams& p, int n, int g
 
 // Initial state of a segment (cold path, kept out of line so the chunk loop stays small): the slot
 // contents (or zero) pushed through the summaries of the earlier segments, S <- A_j S + U_j; writes the bf16
-// copy for the readout and a_0 S for the first update.  One thread = one d_v lane of one state.
+// copy for the readout and a_0 S for the first update.  One thread = one d_v lane of one state and the d_k rows
+// 32 bt_begin .. 32 bt_end - 1.  The fold is a chain of dependent rounds of loads (about a microsecond per earlier
+// segment for one warp per lane quadrant), so when there is something to load the tile warp of the same quadrant,
+// which would otherwise wait for the first tiles, takes half of the rows.
 __device__ __noinline__ void init_state_pass(const float* base, int use_initial_state, const float* wsu, int g, int hi, int v,
-                                             float a, uint32_t s_addr, uint32_t sb_addr) {
+                                             float a, uint32_t s_addr, uint32_t sb_addr, int bt_begin, int bt_end) {
 #pragma unroll 1
-    for (int bt = 0; bt < 4; ++bt) {
+    for (int bt = bt_begin; bt < bt_end; ++bt) {
         float acc[32];
 #pragma unroll
         for (int k = 0; k < 32; ++k) acc[k] = use_initial_state ? base[(size_t)(32 * bt + k) * D + v] : 0.f;
@@ -243,6 +246,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int nc = sq.c_end - sq.c_begin;
     const int t0 = sq.t_begin + sq.c_begin * C;   // first token of this segment
     const int tok0 = sq.c_begin * C;              // its index inside the sequence
+    const bool init_shared = (g > 0 && tp.ws) || p.use_initial_state;   // the initial state is loaded, not just zero
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch behind this grid (the decode step) may be scheduled early
     TL_INIT;
     if (tid == 0) TL(0, 63, 6);
@@ -254,6 +258,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         for (int i = 0; i < 3; ++i) { mbar_init(&sh.kq_full[i], 1); mbar_init(&sh.kq_empty[i], 2); }   // both issuers release a buffer
         for (int i = 0; i < 2; ++i) { mbar_init(&sh.v_full[i], 1); mbar_init(&sh.x_empty[i], 2); }
         mbar_init(&sh.pt_free, 1);
+        mbar_init(&sh.init_done, 8);     // the tile warps' share of the initial state
         mbar_init(&sh.p_full[0], 1); mbar_init(&sh.p_free, 8);   // every tile warp passes p_full before P is overwritten
         mbar_init(&sh.prep_ready[0], 8);
         mbar_init(&sh.sb_ready[0], 4); mbar_init(&sh.sb_ready[1], 4); mbar_init(&sh.s_ready[0], 4); mbar_init(&sh.s_ready[1], 4);
@@ -414,6 +419,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
 
         int k3 = 0, ph3 = 0;      // c mod 3, parity of c / 3
+        if (init_shared) {
+            // rows 64..127 of the initial state of state `half` for this lane quadrant, while the first tiles are in flight
+            const float* gsrc = half == 0 ? p.g_hist : p.g_rec;
+            float a0 = fmaxf(load_gate(gsrc, t0 + 2 * lane, p.H, h, tok0 + 2 * lane < sq.len), 0.f) *
+                       fmaxf(load_gate(gsrc, t0 + 2 * lane + 1, p.H, h, tok0 + 2 * lane + 1 < sq.len), 0.f);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) a0 *= __shfl_xor_sync(0xffffffffu, a0, off);      // decay of chunk 0
+            if (g > 0 && tp.ws) asm volatile("griddepcontrol.wait;" ::: "memory");
+            init_state_pass(slot1 + (size_t)half * state_stride, p.use_initial_state,
+                            tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, half, 32 * q + lane, a0,
+                            lane_addr + COL_S + 128 * half, lane_addr + COL_SB + 64 * half, 2, 4);
+            tc_wait_st();
+            tc_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.init_done);
         for (int c = 0; c < nc; ++c, k3 = k3 == 2 ? 0 : k3 + 1, ph3 ^= (k3 == 0)) {
             const int s = c & 1;
             GateSmem& gs = sh.gs[s];
@@ -620,8 +641,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // everything up to here (and all of chunk 0's operand work in the other warps) is independent of it.
                 if (g > 0 && tp.ws) asm volatile("griddepcontrol.wait;" ::: "memory");
                 init_state_pass(slot1 + (size_t)hi * state_stride, p.use_initial_state,
-                                tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, hi, v, a, s_addr, sb_addr);
+                                tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, hi, v, a, s_addr, sb_addr,
+                                0, init_shared ? 2 : 4);
                 tc_wait_st();
+                mbar_wait(&sh.init_done, 0, abortp, p.status);     // the other half (or nothing) from the tile warps
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.sb_ready[hi]); mbar_arrive(&sh.s_ready[hi]); }
