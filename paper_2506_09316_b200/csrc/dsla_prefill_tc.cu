@@ -522,10 +522,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         auto fetch = [&](int c, float2& lo, float2& hi2) {
             const int j = c * C + lane;
             const bool in = c < nc;
-            lo.x = fmaxf(load_gate(p.g_hist, t0 + j, p.H, h, in && tok0 + j < sq.len), 0.f);
-            lo.y = fmaxf(load_gate(p.g_rec, t0 + j, p.H, h, in && tok0 + j < sq.len), 0.f);
-            hi2.x = fmaxf(load_gate(p.g_hist, t0 + j + 32, p.H, h, in && tok0 + j + 32 < sq.len), 0.f);
-            hi2.y = fmaxf(load_gate(p.g_rec, t0 + j + 32, p.H, h, in && tok0 + j + 32 < sq.len), 0.f);
+            // raw values: nothing may consume them here, or the warp would sit out the load latency in every chunk
+            lo.x = load_gate(p.g_hist, t0 + j, p.H, h, in && tok0 + j < sq.len);
+            lo.y = load_gate(p.g_rec, t0 + j, p.H, h, in && tok0 + j < sq.len);
+            hi2.x = load_gate(p.g_hist, t0 + j + 32, p.H, h, in && tok0 + j + 32 < sq.len);
+            hi2.y = load_gate(p.g_rec, t0 + j + 32, p.H, h, in && tok0 + j + 32 < sq.len);
         };
         float2 nlo, nhi;
         fetch(0, nlo, nhi);
@@ -533,7 +534,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int s = c & 1;
             GateSmem& gs = sh.gs[s];
             __nv_bfloat16* Mm = reinterpret_cast<__nv_bfloat16*>(tiles + OFF_MASK + s * MASK_BYTES);
-            const float2 glo = nlo, ghi = nhi;
+            const float2 glo = make_float2(fmaxf(nlo.x, 0.f), fmaxf(nlo.y, 0.f)), ghi = make_float2(fmaxf(nhi.x, 0.f), fmaxf(nhi.y, 0.f));
             fetch(c + 1, nlo, nhi);
             TLT(tlg0);
             float l1a = warp_prefix_sum(lg2_gate(glo.x), lane), l2a = warp_prefix_sum(lg2_gate(glo.y), lane);
@@ -824,15 +825,15 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
         const int i = warp - 10;
         const float* gsrc = i == 0 ? p.g_hist : p.g_rec;
         float R = 1.f;                                 // product of the gates of all later chunks
-        float n0 = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane, p.H, h, true), 0.f);
-        float n1 = fmaxf(load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane + 1, p.H, h, true), 0.f);
+        float n0 = load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane, p.H, h, true);     // raw; clamped where it is used
+        float n1 = load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane + 1, p.H, h, true);
         for (int it = 0; it < nc; ++it) {
             const int s = it % SUM_STAGES, u = it / SUM_STAGES;
-            const float g0 = n0, g1 = n1;
+            const float g0 = fmaxf(n0, 0.f), g1 = fmaxf(n1, 0.f);
             if (it + 1 < nc) {
                 const int t = t0 + (nc - 2 - it) * C + 2 * lane;
-                n0 = fmaxf(load_gate(gsrc, t, p.H, h, true), 0.f);
-                n1 = fmaxf(load_gate(gsrc, t + 1, p.H, h, true), 0.f);
+                n0 = load_gate(gsrc, t, p.H, h, true);      // consumed in the next iteration
+                n1 = load_gate(gsrc, t + 1, p.H, h, true);
             }
             if (it + 1 + SUM_GATE_AHEAD < nc) {
                 // One chunk of look-ahead does not cover the DRAM latency (this warp's iteration is shorter): pull the gates
