@@ -122,7 +122,10 @@ def barrier(world):
         dist.barrier()
 
 
-def workload_spec(name):
+def workload_spec(name, dense=None):
+    if dense:      # "B,H,T": a dense bf16 batch of the cfg2 head size, for shape sweeps (parity tests cover such shapes)
+        B, H, T = (int(x) for x in dense.split(","))
+        return dict(seed=1900, B=B, H=H, d=128, T=T, dtype="bf16", chunk=64, lens=[T] * B)
     c = dict(gen.CONFIGS[name])
     if name in ("cfg2", "cfg3"):
         c["lens"] = [c["T"]] * c["B"]
@@ -143,7 +146,7 @@ def bench_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
-    spec = workload_spec(args.workload)
+    spec = workload_spec(args.workload, args.dense)
     H, d, lens = spec["H"], spec["d"], spec["lens"]
     N, T_total, max_len = len(lens), int(sum(lens)), int(max(lens))
     dense = len(set(lens)) == 1
@@ -203,7 +206,7 @@ def bench_ours(args):
     flops = T_total * H * FLOP_PER_TOKEN_HEAD(d, 64)
     achieved_tf = flops / (prefill_ms * 1e-3) / 1e12
     # DRAM bytes per prefill from the ncu capture summarised in profiles/prefill_tc_cfg2.md (main + summary kernel)
-    traffic = 181.0e6 if (args.workload == "cfg2" and args.kernel != "simt") else None
+    traffic = 181.0e6 if (args.workload == "cfg2" and not args.dense and args.kernel != "simt") else None
     roofline = {"kernel": "prefill (summary + main launch)", "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"], "traffic": traffic,
                 "algorithmic_bytes": bytes_per_set, "algorithmic_flops": flops,
@@ -229,7 +232,7 @@ def bench_ours(args):
             "metric": "dsla_prefill_plus_decode_tokens_per_s", "value": value, "unit": "tokens/s (one layer)",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{args.workload}: DSLA layer prefill B={N} H={H} d={d} T={lens[0] if dense else 'ragged'} "
+            "config": {"workload": f"{'dense ' + args.dense if args.dense else args.workload}: DSLA layer prefill B={N} H={H} d={d} T={lens[0] if dense else 'ragged'} "
                                    f"(T_total={T_total}) bf16 chunk=64 + 1 decode token per sequence",
                        "kernel": args.kernel, "l2": f"rotating {n_sets} input sets ({n_sets * bytes_per_set / 1e6:.0f} MB > 126 MB L2)",
                        "parallelism": f"replicated x{world} (independent sequences, no collective)"},
@@ -354,7 +357,7 @@ def bench_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    spec = workload_spec(args.workload)
+    spec = workload_spec(args.workload, getattr(args, "dense", None))
     lens = spec["lens"]
     per = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
     res = None
@@ -386,6 +389,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--dense", default=None, metavar="B,H,T", help="shape sweep: a dense bf16 d=128 batch instead of --workload")
     ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-layers", type=int, default=0, help="layers in the decode section (0 = the workload's 32); "
