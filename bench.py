@@ -205,7 +205,7 @@ def bench_ours(args):
 
     flops = T_total * H * FLOP_PER_TOKEN_HEAD(d, 64)
     achieved_tf = flops / (prefill_ms * 1e-3) / 1e12
-    # DRAM bytes per prefill from the ncu capture summarised in profiles/prefill_tc_cfg2.md (main + summary kernel)
+    # DRAM bytes per prefill (main + summary kernel) from one ncu capture of this workload; its summary is kept with the other profiles
     traffic = 181.0e6 if (args.workload == "cfg2" and not args.dense and args.kernel != "simt") else None
     roofline = {"kernel": "prefill (summary + main launch)", "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"], "traffic": traffic,
