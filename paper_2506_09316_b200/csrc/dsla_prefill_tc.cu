@@ -229,9 +229,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const PrefillParams& p = tp.p;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = blockIdx.x % tp.nseg;
-    const int h = (blockIdx.x / tp.nseg) % p.H;
-    const int rank = blockIdx.x / (tp.nseg * p.H);
+    // Blocks are handed out in index order: the last segments first.  When this grid starts as a programmatic dependent
+    // of the summary grid, the blocks that fit next to it are then the ones with the longest fold of summaries ahead of
+    // them, and their prologue (TMEM, first tiles, first scores) is hidden behind the summary grid's tail.
+    const int units = p.N * p.H;
+    const int g = tp.nseg - 1 - (int)(blockIdx.x / units);
+    const int h = (blockIdx.x % units) % p.H;
+    const int rank = (blockIdx.x % units) / p.H;
     const int n = tp.order ? tp.order[rank] : rank;
     const SeqInfo sq = seq_info(p, n, g, tp.nseg, tp.cps, tp.skew8);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
