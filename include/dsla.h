@@ -180,7 +180,11 @@ dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cu
  * (pinned memory gives asynchronous copies); gamma, cu_seqlens, slots and the workspace stay
  * device pointers.  `staging` is caller-owned device memory of at least
  * dsla_*_staging_bytes(a); inputs are copied into it, the kernels run on it, and o is copied back,
- * all on `cuda_stream`.  The caller synchronises the stream before reading o.
+ * all ordered on `cuda_stream`.  The caller synchronises the stream before reading o.  A single dense sequence of
+ * 2048 tokens or more (cu_seqlens == NULL, N == 1) is cut into slices of about 1024 tokens: while slice i is computed,
+ * continuing from the states slice i-1 left in the slot, the inputs of slice i+1 and the outputs of slice i-1 are copied
+ * on two internal streams (created once per device) that are forked from and joined back into `cuda_stream` with
+ * events; the result equals the unsliced one up to floating-point summation order.
  * ------------------------------------------------------------------------------------------ */
 size_t dsla_prefill_staging_bytes(const dsla_prefill_args* a);
 dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* staging,

@@ -1,5 +1,6 @@
 // C-ABI entry points of libdsla: argument checks, state store management, kernel dispatch.
 #include <atomic>
+#include <mutex>
 #include <cstdio>
 #include <cstdlib>
 #include <new>
@@ -228,6 +229,77 @@ size_t dsla_prefill_staging_bytes(const dsla_prefill_args* a) {
     return 4 * t + 2 * g;
 }
 
+// Side streams and events of the host-buffer prefill pipeline, one set per device, created on first use and kept.
+namespace {
+constexpr int HOST_MAX_SLICES = 8;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t start = nullptr, end = nullptr, copied[HOST_MAX_SLICES] = {}, done[HOST_MAX_SLICES] = {};
+};
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[64];
+
+HostPipe* host_pipe() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe& hp = g_pipes[dev];
+    if (!hp.ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp.end, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < HOST_MAX_SLICES; ++i)
+            ok = cudaEventCreateWithFlags(&hp.copied[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { (void)cudaGetLastError(); return nullptr; }
+        hp.ready = true;
+    }
+    return &hp;
+}
+
+// One long sequence from host buffers: the tokens are cut into slices, and while slice i is being computed (continuing
+// from the states slice i-1 left in the slot) slice i+1 is on its way to the device and the outputs of slice i-1 are on
+// their way back, on two side streams that are forked from and joined back into the caller's stream with events.
+dsla_status prefill_host_sliced(const dsla_prefill_args* a, const dsla_prefill_args& d, dsla_state* st, cudaStream_t s) {
+    HostPipe* hp = host_pipe();
+    if (!hp) return DSLA_ERR_CUDA;
+    const int T = a->T_total;
+    int nsl = T / 1024;
+    if (nsl > HOST_MAX_SLICES) nsl = HOST_MAX_SLICES;
+    const int per = ((T + nsl - 1) / nsl + 63) / 64 * 64;          // whole chunks per slice
+    const size_t row = (size_t)a->H * a->d_k * esize(a->dtype), grow = (size_t)a->H * sizeof(float);
+    bool ok = cudaEventRecord(hp->start, s) == cudaSuccess && cudaStreamWaitEvent(hp->h2d, hp->start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(hp->d2h, hp->start, 0) == cudaSuccess;
+    int used = 0;
+    for (int i = 0, t0 = 0; ok && t0 < T; ++i, t0 += per, ++used) {
+        const int len = T - t0 < per ? T - t0 : per;
+        const size_t off = (size_t)t0 * row, goff = (size_t)t0 * grow, nb = (size_t)len * row, ngb = (size_t)len * grow;
+        auto dev = [&](const void* p, size_t o) { return const_cast<char*>(static_cast<const char*>(p)) + o; };
+        ok = cudaMemcpyAsync(dev(d.q, off), dev(a->q, off), nb, cudaMemcpyHostToDevice, hp->h2d) == cudaSuccess &&
+             cudaMemcpyAsync(dev(d.k, off), dev(a->k, off), nb, cudaMemcpyHostToDevice, hp->h2d) == cudaSuccess &&
+             cudaMemcpyAsync(dev(d.v, off), dev(a->v, off), nb, cudaMemcpyHostToDevice, hp->h2d) == cudaSuccess &&
+             cudaMemcpyAsync(dev(d.g_hist, goff), dev(a->g_hist, goff), ngb, cudaMemcpyHostToDevice, hp->h2d) == cudaSuccess &&
+             cudaMemcpyAsync(dev(d.g_rec, goff), dev(a->g_rec, goff), ngb, cudaMemcpyHostToDevice, hp->h2d) == cudaSuccess &&
+             cudaEventRecord(hp->copied[i], hp->h2d) == cudaSuccess && cudaStreamWaitEvent(s, hp->copied[i], 0) == cudaSuccess;
+        if (!ok) break;
+        dsla_prefill_args sl = d;
+        sl.q = dev(d.q, off); sl.k = dev(d.k, off); sl.v = dev(d.v, off); sl.o = dev(d.o, off);
+        sl.g_hist = reinterpret_cast<const float*>(dev(d.g_hist, goff));
+        sl.g_rec = reinterpret_cast<const float*>(dev(d.g_rec, goff));
+        sl.T = len; sl.T_total = len; sl.max_seqlen = len;
+        sl.use_initial_state = i > 0 ? 1 : a->use_initial_state;
+        const dsla_status rc = prefill_device(&sl, st, s);
+        if (rc != DSLA_OK) return rc;
+        ok = cudaEventRecord(hp->done[i], s) == cudaSuccess && cudaStreamWaitEvent(hp->d2h, hp->done[i], 0) == cudaSuccess &&
+             cudaMemcpyAsync(dev(a->o, off), dev(d.o, off), nb, cudaMemcpyDeviceToHost, hp->d2h) == cudaSuccess;
+    }
+    ok = ok && cudaEventRecord(hp->end, hp->d2h) == cudaSuccess && cudaStreamWaitEvent(s, hp->end, 0) == cudaSuccess;
+    return ok ? DSLA_OK : DSLA_ERR_CUDA;
+}
+}  // namespace
+
 dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* staging, size_t staging_bytes, void* cuda_stream) {
     dsla_status rc = check_prefill_sizes(a);
     if (rc != DSLA_OK) return rc;
@@ -243,6 +315,7 @@ dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* 
     d.q = base; d.k = base + t; d.v = base + 2 * t; d.o = base + 3 * t;
     d.g_hist = reinterpret_cast<float*>(base + 4 * t);
     d.g_rec = reinterpret_cast<float*>(base + 4 * t + g);
+    if (a->cu_seqlens == nullptr && a->N == 1 && a->T_total >= 2048) return prefill_host_sliced(a, d, st, s);
     bool ok = cudaMemcpyAsync(const_cast<void*>(d.q), a->q, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(const_cast<void*>(d.k), a->k, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(const_cast<void*>(d.v), a->v, tb, cudaMemcpyHostToDevice, s) == cudaSuccess;
