@@ -21,38 +21,83 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Non-blocking test of a phase (mbarrier.try_wait would park the thread for a while before it reports "not yet").
-__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
+// (waits poll with mbarrier.test_wait: mbarrier.try_wait would park the thread for a while before it reports "not yet")
 
 // Bounded wait.  The fast path (phase already complete) is a single inlined test; otherwise a
 // non-inlined loop polls with a short sleep between tests.  It gives up after `limit` polls, raises
-// *abort_flag (shared) and *status (global) and returns false.  Once the
-// abort flag is up every later wait returns at once, so a CTA that lost a signal still runs to
-// its end, frees its TMEM and exits instead of hanging.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    constexpr uint32_t limit = 4000000u;   // polls of a hundred nanoseconds or more each: about a second
+// *abort_flag (shared) and *status (global) and returns false.  Once the abort flag is up every
+// later wait returns on its first poll, so a CTA that lost a signal still runs to its end, frees its
+// TMEM and exits instead of hanging.  CLUSTER = true makes the successful test an acquire at
+// cluster scope (data another CTA of the cluster wrote into this CTA's shared memory before its
+// remote arrive is then visible).
+constexpr uint32_t MBAR_WAIT_LIMIT = 4000000u;   // polls of a hundred nanoseconds or more each: about a second
+
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_test_wait_t(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    if (CLUSTER)
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+    else
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity)
+            : "memory");
+    return ok != 0;
+}
+template <bool CLUSTER>
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, uint32_t limit) {
     for (uint32_t i = 0; i < limit; ++i) {
-        if (mbar_test_wait(bar, parity)) return true;
+        if (mbar_test_wait_t<CLUSTER>(bar, parity)) return true;
+        if ((i & 63u) == 0u && *abort_flag) return false;
         __nanosleep(100);  // a hot spin takes issue slots from the warps that are doing the work (measured: +4 % run time);
                            // sleeps of 20..400 ns are equal within noise, 1 us costs 10 %
-        if ((i & 1023u) == 1023u && *abort_flag) return false;
     }
     *abort_flag = 1;
     atomicExch(status, 5 /* DSLA_ERR_TIMEOUT */);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (mbar_test_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status);
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          uint32_t limit = MBAR_WAIT_LIMIT) {
+    if (mbar_test_wait_t<false>(bar, parity)) return true;
+    return mbar_wait_slow<false>(bar, parity, abort_flag, status, limit);
 }
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                  uint32_t limit = MBAR_WAIT_LIMIT) {
+    if (mbar_test_wait_t<true>(bar, parity)) return true;
+    return mbar_wait_slow<true>(bar, parity, abort_flag, status, limit);
+}
+
+// ---- thread-block cluster: ranks, barrier, the peer CTA's shared memory ---------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Every thread of the CTA executes both (a full barrier over all threads of the cluster).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in the CTA of the given rank (shared::cluster window).
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32x4(uint32_t caddr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+// Arrive on an mbarrier in another CTA of the cluster; release at cluster scope orders this thread's earlier
+// writes (and, after a __syncwarp, those of its warp) before the arrival.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(caddr) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
