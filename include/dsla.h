@@ -75,9 +75,18 @@ void* dsla_state_data(dsla_state* st);
  * store when slots_dev == NULL (n is then ignored). */
 dsla_status dsla_state_zero(dsla_state* st, const int32_t* slots_dev, int n, void* cuda_stream);
 
-/* Reads back (synchronising the whole device) and clears the status word that kernels set when a
- * bounded wait gives up: DSLA_OK or DSLA_ERR_TIMEOUT. */
+/* Reads back (synchronising the whole device) and clears the status word that kernels raise for problems only the
+ * device can see: DSLA_OK; DSLA_ERR_TIMEOUT when a bounded on-device wait gave up (the kernel then ran to its end
+ * without hanging, its results are invalid); DSLA_ERR_INVALID_ARG when a packed sequence turned out longer than
+ * max_seqlen (the tensor-core prefill sizes its segments from max_seqlen, so the tail of that sequence was not
+ * computed). */
 dsla_status dsla_state_last_error(dsla_state* st);
+
+/* Diagnostic: exercises the give-up path of the bounded waits without hanging anything.  A one-warp kernel waits,
+ * for at most max_polls polls (1 .. 1,000,000; a poll takes about 0.1 us), on a barrier that nobody arrives at; the
+ * wait runs out, the kernel raises the status word of `st` and returns.  dsla_state_last_error(st) then reports
+ * DSLA_ERR_TIMEOUT and the device stays usable.  (No counterpart in the paper.) */
+dsla_status dsla_selftest_bounded_wait(dsla_state* st, unsigned max_polls, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Prefill: the chunkwise-parallel form of the recurrence.  Inside a chunk of C tokens the output

@@ -62,6 +62,8 @@ _lib.dsla_state_zero.argtypes = [c_void_p, c_void_p, c_int, c_void_p]
 _lib.dsla_state_zero.restype = c_int
 _lib.dsla_state_last_error.argtypes = [c_void_p]
 _lib.dsla_state_last_error.restype = c_int
+_lib.dsla_selftest_bounded_wait.argtypes = [c_void_p, ctypes.c_uint, c_void_p]
+_lib.dsla_selftest_bounded_wait.restype = c_int
 _lib.dsla_prefill_workspace_bytes.argtypes = [POINTER(dsla_prefill_args)]
 _lib.dsla_prefill_workspace_bytes.restype = c_size_t
 _lib.dsla_prefill.argtypes = [POINTER(dsla_prefill_args), c_void_p, c_void_p]
@@ -127,10 +129,14 @@ class DslaState:
             pass
 
 
-def dsla_state_alloc(num_slots: int, H: int, d_k: int, d_v: int, device="cuda") -> DslaState:
-    """The store borrows a torch allocation, so the library itself calls no cudaMalloc for it."""
+def dsla_state_alloc(num_slots: int, H: int, d_k: int, d_v: int, device="cuda", buffer=None) -> DslaState:
+    """The store borrows a torch allocation, so the library itself calls no cudaMalloc for it.  ``buffer`` may be a
+    contiguous fp32 tensor of the store's size that the caller owns (e.g. a view into a larger allocation)."""
     n = dsla_state_bytes(num_slots, H, d_k, d_v)
-    buf = torch.empty((num_slots, 2, H, d_k, d_v), dtype=torch.float32, device=device) if n else None
+    if buffer is not None:
+        buf = buffer.view(num_slots, 2, H, d_k, d_v)
+    else:
+        buf = torch.empty((num_slots, 2, H, d_k, d_v), dtype=torch.float32, device=device) if n else None
     h = c_void_p()
     with torch.cuda.device(buf.device if buf is not None else device):
         rc = _lib.dsla_state_alloc(byref(h), num_slots, H, d_k, d_v, _ptr(buf), n)
@@ -155,6 +161,10 @@ def dsla_state_zero(st: DslaState, slots=None, stream=None):
 
 def dsla_state_last_error(st: DslaState) -> int:
     return int(_lib.dsla_state_last_error(st.handle))
+
+
+def dsla_selftest_bounded_wait(st: DslaState, max_polls: int = 2000, stream=None):
+    _check(_lib.dsla_selftest_bounded_wait(st.handle, int(max_polls), _stream(stream)), "dsla_selftest_bounded_wait")
 
 
 def _prefill_args(q, k, v, o, g_hist, g_rec, gamma, cu_seqlens, slots, N, T, max_seqlen, chunk, scale,

@@ -114,7 +114,14 @@ dsla_status dsla_state_last_error(dsla_state* st) {
     if (cudaDeviceSynchronize() != cudaSuccess) return DSLA_ERR_CUDA;
     if (cudaMemcpy(&host, st->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return DSLA_ERR_CUDA;
     if (host != 0 && cudaMemset(st->status, 0, sizeof(int)) != cudaSuccess) return DSLA_ERR_CUDA;
-    return host == 0 ? DSLA_OK : DSLA_ERR_TIMEOUT;
+    if (host == 0) return DSLA_OK;
+    return host == (int)DSLA_ERR_INVALID_ARG ? DSLA_ERR_INVALID_ARG : DSLA_ERR_TIMEOUT;
+}
+
+dsla_status dsla_selftest_bounded_wait(dsla_state* st, unsigned max_polls, void* cuda_stream) {
+    if (!st || max_polls == 0 || max_polls > 1000000u) return DSLA_ERR_INVALID_ARG;
+    launch_bounded_wait_selftest(st->status, max_polls, static_cast<cudaStream_t>(cuda_stream));
+    return cudaGetLastError() == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
 }
 
 // ---- prefill ------------------------------------------------------------------------------

@@ -49,6 +49,8 @@ dsla_status prefill_checked(const dsla_prefill_args* a, dsla_state* st, cudaStre
 dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStream_t s);
 // dsla_prefill_simt.cu
 dsla_status launch_prefill_simt(const PrefillParams& p, int d, int chunk, dsla_dtype dt, cudaStream_t s);
+// dsla_prefill_summary.cu: one warp waits, with the given poll limit, on a barrier nobody arrives at
+void launch_bounded_wait_selftest(int* status, unsigned max_polls, cudaStream_t s);
 // dsla_prefill_tc.cu
 bool prefill_tc_available();
 size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a);

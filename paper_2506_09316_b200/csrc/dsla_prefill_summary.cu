@@ -196,6 +196,24 @@ __global__ void __launch_bounds__(256) state_snapshot_kernel(const PrefillParams
     for (int k = threadIdx.x; k < D * D / 4; k += 256) dst[k] = src[k];
 }
 
+// The give-up path of the bounded waits, on its own: one warp, one barrier that nobody ever arrives at, nothing
+// asynchronous in flight.  The wait runs out after max_polls polls, raises the status word and the kernel returns.
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(int* status, unsigned max_polls) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncwarp();
+    volatile int* abortp = &abort_flag;
+    if (threadIdx.x == 0) mbar_wait(&bar, 0, abortp, status, max_polls);
+    __syncwarp();
+    // a wait that starts after the abort flag is up returns on its first poll
+    mbar_wait(&bar, 0, abortp, status, MBAR_WAIT_LIMIT);
+}
+
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -229,6 +247,11 @@ bool make_tile_map(CUtensorMap* m, const void* base, int T_total, int H) {
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+void launch_bounded_wait_selftest(int* status, unsigned max_polls, cudaStream_t s) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(status, max_polls);
+    count_launch();
 }
 
 void launch_seq_order(const int32_t* cu, int N, int* order, cudaStream_t s) {

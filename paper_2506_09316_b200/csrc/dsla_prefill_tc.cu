@@ -69,8 +69,6 @@ struct alignas(16) GateA {
 // Factors of a chunk whose local part this CTA computes (both states).
 struct alignas(16) GateB {
     float L[2][C];            // cumulative log2-gates
-    float f[2][32];           // 2^(L_31 - L_s), s < 32         (column factors of the block rows 32.., columns ..31)
-    float e[2][32];           // W_i 2^(L_j - L_31), j >= 32     (row factors of that block)
 };
 
 struct alignas(16) Shared {
@@ -79,7 +77,7 @@ struct alignas(16) Shared {
     uint64_t vt_ready[2], vt_free[2];
     uint64_t s_ready, sb_ready, u_full, o_full, o_free;
     uint64_t p_full, p_free, pt_ready, pt_free, oi_full, oi_free;
-    uint64_t x_full[2][4], x_free[2][4];
+    uint64_t x_full[2][4];
     uint32_t tmem_base;
     int abort_flag;
     GateA ga[NGA];
@@ -109,6 +107,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     // Every early exit below depends only on values both CTAs of the cluster share, and comes before any cluster
     // operation.
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
+    // A sequence longer than the max_seqlen the host sized the segments for would lose its tail: say so.
+    if (tid == 0 && g == 0 && sq.nchunks > seg_begin(tp.nseg, tp.nseg, tp.cps, tp.skew8)) atomicExch(p.status, (int)DSLA_ERR_INVALID_ARG);
     const size_t state_stride = (size_t)p.H * D * D;
     float* slot_i = p.state + (((size_t)sq.slot * 2 + rank) * p.H + h) * (size_t)(D * D);
     if (sq.len <= 0) {  // empty sequence: a fresh start leaves zero states, a resume leaves the slot alone
@@ -133,7 +133,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(&sh.p_full, 1); mbar_init(&sh.p_free, 4); mbar_init(&sh.pt_ready, 4); mbar_init(&sh.pt_free, 1);
         mbar_init(&sh.oi_full, 1); mbar_init(&sh.oi_free, 4);
         for (int b = 0; b < 2; ++b)
-            for (int q = 0; q < 4; ++q) { mbar_init(&sh.x_full[b][q], 1); mbar_init(&sh.x_free[b][q], 1); }
+            for (int q = 0; q < 4; ++q) mbar_init(&sh.x_full[b][q], 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -185,24 +185,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_commit(&sh.p_full);
             };
             for (int c = 0; c < NST && c < nc; ++c) load(c);
-            if (rank == 0) scores(0);
 #pragma unroll 1
-            for (int c = 0; c < nc; ++c) {
-                const int s = c % NST, b = c & 1;
-                if (c >= 1 && c + 2 < nc) {      // the stage of chunk c - 1 takes chunk c + 2
-                    WAIT(&sh.ld_empty[(c - 1) % NST], ((c - 1) / NST) & 1);
-                    load(c + 2);
-                }
-                WAIT(&sh.ld_full[s], (c / NST) & 1);
-                WAIT(&sh.vt_ready[b], (c >> 1) & 1);
-                WAIT(&sh.s_ready, c & 1);
-                tc_fence_after();
-                const uint64_t bk = dk_n + (uint64_t)s * ST_STEP;
+            for (int c = -1; c < nc; ++c) {        // iteration -1 only issues the scores of chunk 0
+                if (c >= 0) {
+                    const int s = c % NST, b = c & 1;
+                    if (c >= 1 && c + 2 < nc) {      // the stage of chunk c - 1 takes chunk c + 2
+                        WAIT(&sh.ld_empty[(c - 1) % NST], ((c - 1) / NST) & 1);
+                        load(c + 2);
+                    }
+                    WAIT(&sh.ld_full[s], (c / NST) & 1);
+                    WAIT(&sh.vt_ready[b], (c >> 1) & 1);
+                    WAIT(&sh.s_ready, c & 1);
+                    tc_fence_after();
+                    const uint64_t bk = dk_n + (uint64_t)s * ST_STEP;
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_S, tb + COL_VT + 32 * b + 8 * kk, bk + (uint64_t)(kk * 128), ID_D, 1);
-                tc_commit(&sh.u_full);
-                tc_commit(&sh.vt_free[b]);
-                tc_commit(&sh.ld_empty[s]);
+                    for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_S, tb + COL_VT + 32 * b + 8 * kk, bk + (uint64_t)(kk * 128), ID_D, 1);
+                    tc_commit(&sh.u_full);
+                    tc_commit(&sh.vt_free[b]);
+                    tc_commit(&sh.ld_empty[s]);
+                }
                 if (c + 1 < nc && ((c + 1) & 1) == rank) scores(c + 1);
             }
         }
@@ -297,15 +298,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 float ma = warp_prefix_sum(lg2_gate(gx_lo), lane), mb = warp_prefix_sum(lg2_gate(gx_hi), lane);
                 const float midx = __shfl_sync(0xffffffffu, ma, 31);
                 mb += midx;
-                const float l1a = rank == 0 ? la : ma, l1b = rank == 0 ? lb : mb, mid1 = rank == 0 ? mid : midx;
-                const float l2a = rank == 0 ? ma : la, l2b = rank == 0 ? mb : lb, mid2 = rank == 0 ? midx : mid;
+                const float l1a = rank == 0 ? la : ma, l1b = rank == 0 ? lb : mb;
+                const float l2a = rank == 0 ? ma : la, l2b = rank == 0 ? mb : lb;
                 if (nb >= NGB) WAIT(&sh.gb_empty[kb], ((nb / NGB) - 1) & 1);
                 GateB& gb = sh.gb[kb];
                 gb.L[0][lane] = l1a; gb.L[0][lane + 32] = l1b;
                 gb.L[1][lane] = l2a; gb.L[1][lane + 32] = l2b;
-                // the block of rows 32..63 and columns 0..31 factors through token 31, both factors <= 1
-                gb.f[0][lane] = ex2(mid1 - l1a); gb.f[1][lane] = ex2(mid2 - l2a);
-                gb.e[0][lane] = W1 * ex2(l1b - mid1); gb.e[1][lane] = W2 * ex2(l2b - mid2);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.gb_full[kb]);
                 ++nb;
@@ -327,56 +325,36 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 WAIT(&sh.gb_full[n2 & (NGB - 1)], (n2 / NGB) & 1);
                 WAIT(&sh.p_full, n2 & 1);
                 tc_fence_after();
-                uint32_t r[32];
-                if (half <= q) { tmem_ld32(lane_addr + COL_P + 32 * half, r); tc_wait_ld(); }
+                if (n2 >= 1) WAIT(&sh.pt_free, (n2 - 1) & 1);       // the previous P~ has been consumed
+                // M[j][s] = W1 2^(L1_j - L1_s) + W2 2^(L2_j - L2_s) for s <= j (differences of logs, never positive), else 0;
+                // eight columns per round, loop kept rolled (the code of all roles has to stay small)
+                const float L1j = gb.L[0][j], L2j = gb.L[1][j];
+#pragma unroll 1
+                for (int m4 = 0; m4 < 4; ++m4) {
+                    const int col0 = 32 * half + 8 * m4;
+                    uint32_t pk[4] = {0u, 0u, 0u, 0u};
+                    if (half <= q) {        // warp-uniform: the block above the diagonal is all zeros
+                        uint32_t r[8];
+                        tmem_ld8(lane_addr + COL_P + col0, r);
+                        const float4 a0 = *reinterpret_cast<const float4*>(&gb.L[0][col0]), a1 = *reinterpret_cast<const float4*>(&gb.L[0][col0 + 4]);
+                        const float4 b0 = *reinterpret_cast<const float4*>(&gb.L[1][col0]), b1 = *reinterpret_cast<const float4*>(&gb.L[1][col0 + 4]);
+                        const float s1[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                        const float s2[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                        float m[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float mm = fmaf(W2, ex2(L2j - s2[e]), W1 * ex2(L1j - s1[e]));
+                            m[e] = (col0 + e <= j) ? mm : 0.f;
+                        }
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            pk[e] = pack_bf16(__uint_as_float(r[2 * e]) * m[2 * e], __uint_as_float(r[2 * e + 1]) * m[2 * e + 1]);
+                    }
+                    *reinterpret_cast<uint4*>(pt + sw128_offset(j, col0)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                }
                 __syncwarp();
                 if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
-                if (n2 >= 1) WAIT(&sh.pt_free, (n2 - 1) & 1);       // the previous P~ has been consumed
-                if (half > q) {
-                    // above the diagonal: zeros
-#pragma unroll
-                    for (int m4 = 0; m4 < 4; ++m4) *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 * half + 8 * m4)) = make_uint4(0u, 0u, 0u, 0u);
-                } else if (half < q) {
-                    // full block: M[j][s] = e1_j f1_s + e2_j f2_s
-                    const float e1 = gb.e[0][lane], e2 = gb.e[1][lane];
-#pragma unroll
-                    for (int m4 = 0; m4 < 4; ++m4) {
-                        const float4 fa0 = *reinterpret_cast<const float4*>(&gb.f[0][8 * m4]), fa1 = *reinterpret_cast<const float4*>(&gb.f[0][8 * m4 + 4]);
-                        const float4 fb0 = *reinterpret_cast<const float4*>(&gb.f[1][8 * m4]), fb1 = *reinterpret_cast<const float4*>(&gb.f[1][8 * m4 + 4]);
-                        const float f1[8] = {fa0.x, fa0.y, fa0.z, fa0.w, fa1.x, fa1.y, fa1.z, fa1.w};
-                        const float f2[8] = {fb0.x, fb0.y, fb0.z, fb0.w, fb1.x, fb1.y, fb1.z, fb1.w};
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float m0 = fmaf(e2, f2[2 * e], e1 * f1[2 * e]), m1 = fmaf(e2, f2[2 * e + 1], e1 * f1[2 * e + 1]);
-                            pk[e] = pack_bf16(__uint_as_float(r[8 * m4 + 2 * e]) * m0, __uint_as_float(r[8 * m4 + 2 * e + 1]) * m1);
-                        }
-                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, 8 * m4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
-                } else {
-                    // diagonal block: M[j][s] = W1 2^(L1_j - L1_s) + W2 2^(L2_j - L2_s) for s <= j, from differences of logs
-                    const float L1j = gb.L[0][j], L2j = gb.L[1][j];
-#pragma unroll
-                    for (int m4 = 0; m4 < 4; ++m4) {
-                        uint32_t pk[4] = {0u, 0u, 0u, 0u};
-                        if (8 * m4 <= lane) {
-                            const float4 a0 = *reinterpret_cast<const float4*>(&gb.L[0][32 * q + 8 * m4]), a1 = *reinterpret_cast<const float4*>(&gb.L[0][32 * q + 8 * m4 + 4]);
-                            const float4 b0 = *reinterpret_cast<const float4*>(&gb.L[1][32 * q + 8 * m4]), b1 = *reinterpret_cast<const float4*>(&gb.L[1][32 * q + 8 * m4 + 4]);
-                            const float s1[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-                            const float s2[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                            float m[8];
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const float mm = fmaf(W2, ex2(L2j - s2[e]), W1 * ex2(L1j - s1[e]));
-                                m[e] = (8 * m4 + e <= lane) ? mm : 0.f;
-                            }
-#pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                pk[e] = pack_bf16(__uint_as_float(r[8 * m4 + 2 * e]) * m[2 * e], __uint_as_float(r[8 * m4 + 2 * e + 1]) * m[2 * e + 1]);
-                        }
-                        *reinterpret_cast<uint4*>(pt + sw128_offset(j, 32 * half + 8 * m4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    }
-                }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.pt_ready); mbar_arrive(&sh.gb_empty[n2 & (NGB - 1)]); }
@@ -409,45 +387,29 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (lane == 0) { mbar_arrive(&sh.s_ready); mbar_arrive(&sh.sb_ready); }
                 continue;
             }
-            WAIT(&sh.u_full, (c - 1) & 1);
+            WAIT(&sh.u_full, (c - 1) & 1);      // the update of chunk c - 1 is in the fp32 state
+            WAIT(&sh.o_full, (c - 1) & 1);      // the readout of chunk c - 1 has read the previous bf16 copy
             tc_fence_after();
-            uint32_t pk0[16], pk1[16];
-            {
-                const float2 a2 = make_float2(a, a);
-                uint32_t r0[32];
-                tmem_ld32(s_addr, r0);
+            const float2 a2 = make_float2(a, a);
+#pragma unroll 1
+            for (int i = 0; i < 2; ++i) {
+                uint32_t r0[32], pk[16];
+                tmem_ld32(s_addr + 32 * i, r0);
                 tc_wait_ld();
 #pragma unroll
-                for (int k = 0; k < 16; ++k) pk0[k] = pack_bf16(__uint_as_float(r0[2 * k]), __uint_as_float(r0[2 * k + 1]));
+                for (int k = 0; k < 16; ++k) pk[k] = pack_bf16(__uint_as_float(r0[2 * k]), __uint_as_float(r0[2 * k + 1]));
+                tmem_st16(sb_addr + 16 * i, pk);
 #pragma unroll
                 for (int k = 0; k < 32; k += 2) {
                     const float2 y = __fmul2_rn(make_float2(__uint_as_float(r0[k]), __uint_as_float(r0[k + 1])), a2);
                     r0[k] = __float_as_uint(y.x); r0[k + 1] = __float_as_uint(y.y);
                 }
-                tmem_st32(s_addr, r0);
-                tmem_ld32(s_addr + 32, r0);
-                tc_wait_ld();
-#pragma unroll
-                for (int k = 0; k < 16; ++k) pk1[k] = pack_bf16(__uint_as_float(r0[2 * k]), __uint_as_float(r0[2 * k + 1]));
-#pragma unroll
-                for (int k = 0; k < 32; k += 2) {
-                    const float2 y = __fmul2_rn(make_float2(__uint_as_float(r0[k]), __uint_as_float(r0[k + 1])), a2);
-                    r0[k] = __float_as_uint(y.x); r0[k + 1] = __float_as_uint(y.y);
-                }
-                tmem_st32(s_addr + 32, r0);
+                tmem_st32(s_addr + 32 * i, r0);
             }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.s_ready);            // the update of chunk c may accumulate
-            WAIT(&sh.o_full, (c - 1) & 1);                      // the readout of chunk c - 1 has read the previous bf16 copy
-            tc_fence_after();
-            tmem_st16(sb_addr, pk0);
-            tmem_st16(sb_addr + 16, pk1);
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.sb_ready);
+            if (lane == 0) { mbar_arrive(&sh.s_ready); mbar_arrive(&sh.sb_ready); }
         }
         // ---- final state of this segment
         WAIT(&sh.u_full, (nc - 1) & 1);
@@ -463,119 +425,118 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // register, times the bf16 weights, into TMEM as the A operand.
         const uint32_t vcol = (uint32_t)(v >> 6) * 8192u + (uint32_t)((v & 7) << 1);
         const uint32_t vchunk = (uint32_t)((v & 63) >> 3);
+        const uint32_t vrow = smem_u32(tiles + ST_V) + vcol;     // + stage offset + token * 128 + (swizzled 16-byte piece)
         auto make_vt = [&](int c) {
             const int s = c % NST, b = c & 1;
             WAIT(&sh.ld_full[s], (c / NST) & 1);
             WAIT(&sh.ga_full[c & (NGA - 1)], (c / NGA) & 1);
-            const uint8_t* vb = tiles + s * STAGE_BYTES + ST_V + vcol;
-            const uint4* wq = reinterpret_cast<const uint4*>(sh.ga[c & (NGA - 1)].w);
-            uint32_t pk[32];
-#pragma unroll
-            for (int m = 0; m < 8; ++m) {
-                const uint4 w4 = wq[m];
-                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int s0 = 8 * m + 2 * e;      // tokens s0, s0 + 1 (s0 mod 8 and s0 + 1 mod 8 are compile-time constants)
-                    const uint32_t lo = *reinterpret_cast<const unsigned short*>(vb + s0 * 128 + ((vchunk ^ (uint32_t)(s0 & 7)) << 4));
-                    const uint32_t hi = *reinterpret_cast<const unsigned short*>(vb + (s0 + 1) * 128 + ((vchunk ^ (uint32_t)((s0 + 1) & 7)) << 4));
-                    const uint32_t x = lo | (hi << 16);
-                    const __nv_bfloat162 r2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&x), *reinterpret_cast<const __nv_bfloat162*>(&ww[e]));
-                    pk[4 * m + e] = *reinterpret_cast<const uint32_t*>(&r2);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.ld_empty[s]);          // this warp is done with the stage's V tile
             if (c >= 2) WAIT(&sh.vt_free[b], ((c >> 1) - 1) & 1);  // the update of chunk c - 2 has read this buffer
             tc_fence_after();
-            tmem_st32(lane_addr + COL_VT + 32 * b, pk);
+            const uint32_t vb = vrow + (uint32_t)(s * STAGE_BYTES);
+            const uint4* wq = reinterpret_cast<const uint4*>(sh.ga[c & (NGA - 1)].w);
+            const uint32_t vt = lane_addr + COL_VT + 32 * b;
+#pragma unroll 1
+            for (int m = 0; m < 8; ++m) {          // eight tokens per round, loop kept rolled
+                const uint4 w4 = wq[m];
+                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+                uint32_t raw[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) raw[r] = ld_shared_u16(vb + (uint32_t)(m * 1024 + r * 128) + ((vchunk ^ (uint32_t)r) << 4));
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t x = raw[2 * e] | (raw[2 * e + 1] << 16);
+                    const __nv_bfloat162 r2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&x), *reinterpret_cast<const __nv_bfloat162*>(&ww[e]));
+                    pk[e] = *reinterpret_cast<const uint32_t*>(&r2);
+                }
+                tmem_st4(vt + 4 * m, pk);
+            }
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.vt_ready[b]);
+            if (lane == 0) { mbar_arrive(&sh.vt_ready[b]); mbar_arrive(&sh.ld_empty[s]); }
         };
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
         const uint32_t recv_row = (uint32_t)v * 128u;                        // this thread's row in a receive buffer
-        const uint32_t recv_peer = map_to_cta(smem_u32(tiles + OFF_RECV), (uint32_t)peer);
-        uint32_t xfull_peer[2], xfree_peer[2];
-        for (int b = 0; b < 2; ++b) {
-            xfull_peer[b] = map_to_cta(smem_u32(&sh.x_full[b][q]), (uint32_t)peer);
-            xfree_peer[b] = map_to_cta(smem_u32(&sh.x_free[b][q]), (uint32_t)peer);
-        }
-        // Partial outputs of 32 tokens (columns 32 th .. 32 th + 31 of the accumulators) of chunk c for this thread's d_v lane:
+        const uint32_t recv_peer = map_to_cta(smem_u32(tiles + OFF_RECV), (uint32_t)peer) + recv_row;
+        const uint32_t xfull_peer0 = map_to_cta(smem_u32(&sh.x_full[0][q]), (uint32_t)peer);
+        const uint32_t xfull_peer1 = map_to_cta(smem_u32(&sh.x_full[1][q]), (uint32_t)peer);
+        const uint32_t vsw = (uint32_t)(v & 7);
+        // Partial outputs of 16 tokens (columns col .. col + 15 of the accumulators) of chunk c for this thread's d_v lane:
         // rowf_j (O_a + O_b) [+ O_in]
-        auto partial = [&](int c, int th, float (&x)[32]) {
-            uint32_t ra[32], rb[32];
-            tmem_ld32(lane_addr + COL_OA + 32 * th, ra);
-            tmem_ld32(lane_addr + COL_OB + 32 * th, rb);
-            tc_wait_ld();
-            const float4* rf = reinterpret_cast<const float4*>(sh.ga[c & (NGA - 1)].rowf + 32 * th);
+        auto partial16 = [&](int c, int col, float (&x)[16]) {
+            uint32_t ra[16], rb[16];
+            tmem_ld16(lane_addr + COL_OA + col, ra);
+            tmem_ld16(lane_addr + COL_OB + col, rb);
+            const float4* rf = reinterpret_cast<const float4*>(sh.ga[c & (NGA - 1)].rowf + col);
+            float f[16];
 #pragma unroll
-            for (int m = 0; m < 8; ++m) {
-                const float4 f = rf[m];
-                x[4 * m + 0] = f.x * (__uint_as_float(ra[4 * m + 0]) + __uint_as_float(rb[4 * m + 0]));
-                x[4 * m + 1] = f.y * (__uint_as_float(ra[4 * m + 1]) + __uint_as_float(rb[4 * m + 1]));
-                x[4 * m + 2] = f.z * (__uint_as_float(ra[4 * m + 2]) + __uint_as_float(rb[4 * m + 2]));
-                x[4 * m + 3] = f.w * (__uint_as_float(ra[4 * m + 3]) + __uint_as_float(rb[4 * m + 3]));
-            }
+            for (int m = 0; m < 4; ++m) { const float4 t = rf[m]; f[4 * m] = t.x; f[4 * m + 1] = t.y; f[4 * m + 2] = t.z; f[4 * m + 3] = t.w; }
+            tc_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 16; ++k) x[k] = f[k] * (__uint_as_float(ra[k]) + __uint_as_float(rb[k]));
             if ((c & 1) == rank) {
-                tmem_ld32(lane_addr + COL_OI + 32 * th, ra);
+                tmem_ld16(lane_addr + COL_OI + col, ra);
                 tc_wait_ld();
 #pragma unroll
-                for (int k = 0; k < 32; ++k) x[k] += __uint_as_float(ra[k]);
+                for (int k = 0; k < 16; ++k) x[k] += __uint_as_float(ra[k]);
             }
         };
-        make_vt(0);
 #pragma unroll 1
-        for (int c = 0; c < nc; ++c) {
+        for (int c = -1; c < nc; ++c) {       // iteration -1 only prepares chunk 0
             if (c + 1 < nc) make_vt(c + 1);
+            if (c < 0) continue;
             const int b = c & 1;
             WAIT(&sh.o_full, c & 1);
             if ((c & 1) == rank) WAIT(&sh.oi_full, (c >> 1) & 1);
             tc_fence_after();
-            float x[32];
-            // ---- the peer's 32 tokens: send
-            partial(c, peer, x);
-            if (c >= 2) WAIT(&sh.x_free[b][q], ((c >> 1) - 1) & 1);      // the peer has read what chunk c - 2 left in its buffer
+            // ---- the peer's 32 tokens: send.  Its receive buffer b is free: the peer read what chunk c - 2 left there before it
+            // sent its part of chunk c - 1, which this warp has waited for.  The stores complete on the peer's barrier.
             {
-                const uint32_t dst = recv_peer + (uint32_t)b * RECV_BYTES + recv_row;
+                const uint32_t dst = recv_peer + (uint32_t)b * RECV_BYTES, bar = b ? xfull_peer1 : xfull_peer0;
+#pragma unroll 1
+                for (int i = 0; i < 2; ++i) {
+                    float x[16];
+                    partial16(c, 32 * peer + 16 * i, x);
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    st_cluster_f32x4(dst + (((uint32_t)k ^ (uint32_t)(v & 7)) << 4), x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]);
+                    for (int k = 0; k < 4; ++k)
+                        st_async_f32x4(dst + (((uint32_t)(4 * i + k) ^ vsw) << 4), x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3], bar);
+                }
             }
-            __syncwarp();
-            if (lane == 0) { fence_acq_rel_cluster(); mbar_arrive_cluster(xfull_peer[b]); }
-            // ---- own 32 tokens
-            partial(c, rank, x);
+            // ---- own 32 tokens: add what the peer sent, store
+            if (lane == 0) mbar_arrive_expect_tx(&sh.x_full[b][q], 32 * 128);      // the peer's warp q sends 128 bytes per lane
+            mbar_wait_cluster(&sh.x_full[b][q], (uint32_t)((c >> 1) & 1), abortp, p.status);
+            {
+                const int valid = min(C, sq.len - tok0 - c * C) - 32 * rank;     // tokens of this CTA's half that exist
+                // a thread owns one d_v lane; a warp's store of one token is 64 contiguous bytes (two full sectors)
+                __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * rank) * p.H + h) * D + v;
+                const size_t row = (size_t)p.H * D;
+                const uint8_t* src = tiles + OFF_RECV + b * RECV_BYTES + recv_row;
+#pragma unroll 1
+                for (int i = 0; i < 2; ++i) {
+                    float x[16];
+                    partial16(c, 32 * rank + 16 * i, x);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float4 y = *reinterpret_cast<const float4*>(src + (((uint32_t)(4 * i + k) ^ vsw) << 4));
+                        x[4 * k] += y.x; x[4 * k + 1] += y.y; x[4 * k + 2] += y.z; x[4 * k + 3] += y.w;
+                    }
+                    if (valid >= 16 * i + 16) {
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj) dst[(16 * i + jj) * row] = __float2bfloat16_rn(x[jj]);
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 16; ++jj)
+                            if (16 * i + jj < valid) dst[(16 * i + jj) * row] = __float2bfloat16_rn(x[jj]);
+                    }
+                }
+            }
             __syncwarp();
             if (lane == 0) {
                 tc_fence_before();
                 mbar_arrive(&sh.o_free);
                 if ((c & 1) == rank) mbar_arrive(&sh.oi_free);
                 mbar_arrive(&sh.ga_empty[c & (NGA - 1)]);
-            }
-            mbar_wait_cluster(&sh.x_full[b][q], (uint32_t)((c >> 1) & 1), abortp, p.status);
-            {
-                const uint8_t* src = tiles + OFF_RECV + b * RECV_BYTES + recv_row;
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float4 y = *reinterpret_cast<const float4*>(src + ((k ^ (v & 7)) << 4));
-                    x[4 * k] += y.x; x[4 * k + 1] += y.y; x[4 * k + 2] += y.z; x[4 * k + 3] += y.w;
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(xfree_peer[b]);
-            // a thread owns one d_v lane; a warp's store of one token is 64 contiguous bytes (two full sectors)
-            const int valid = min(C, sq.len - tok0 - c * C) - 32 * rank;     // tokens of this CTA's half that exist
-            __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * rank) * p.H + h) * D + v;
-            const size_t row = (size_t)p.H * D;
-            if (valid >= 32) {
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj) dst[jj * row] = __float2bfloat16_rn(x[jj]);
-            } else {
-#pragma unroll
-                for (int jj = 0; jj < 32; ++jj)
-                    if (jj < valid) dst[jj * row] = __float2bfloat16_rn(x[jj]);
             }
         }
     }

@@ -107,6 +107,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int n = tp.order ? tp.order[rank] : rank;
     const SeqInfo sq = seq_info(p, n, g, tp.nseg, tp.cps, tp.skew8);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
+    if (tid == 0 && g == 0 && sq.nchunks > seg_begin(tp.nseg, tp.nseg, tp.cps, tp.skew8)) atomicExch(p.status, (int)DSLA_ERR_INVALID_ARG);
     float* slot1 = p.state + (((size_t)sq.slot * 2) * p.H + h) * (size_t)(D * D);
     const size_t state_stride = (size_t)p.H * D * D;
     // where the initial state is read: the slot, or the snapshot taken before this grid (split sequences)
