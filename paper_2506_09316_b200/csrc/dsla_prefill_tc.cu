@@ -35,26 +35,26 @@ namespace {
 // four warp schedulers of the SM take the warps of one quadrant each, so every role that works on TMEM has one
 // warp per quadrant:
 //   0, 1, 4, 5 : score tile warps (rows 0..31 / 32..63 of P x column halves): P~ = P (.) decay mask
-//   2          : TMA producer; issues the state update and the scores
-//   3          : issues the readout and the chunk-local output; allocates TMEM
+//   2          : TMA producer; issues the state update
+//   3          : issues the readout; allocates TMEM
+//   7          : issues the chunk-local MMAs (scores, O_in)
 //   6          : gate warp (cumulative log-gates and everything derived from them)
 //   8..15      : state warps (two per quadrant, 64 d_k columns each): rescale + bf16 copy of the state
 //   16..19     : V~ into TMEM, then the outputs (scale, exchange with the peer CTA, store)
-constexpr int WARP_X = 2, WARP_Y = 3, WARP_GATE = 6, STATE_W0 = 8, VE_W0 = 16;
-constexpr int NTHREADS = 20 * 32;
+constexpr int WARP_X = 2, WARP_Y = 3, WARP_GATE = 6, WARP_Z = 7, STATE_W0 = 8, VE_W0 = 16;
+constexpr int NTHREADS = 24 * 32;
 constexpr int NST = 3;                             // landing stages of {K, Q, V}
 constexpr int STAGE_BYTES = 3 * 16384, ST_Q = 16384, ST_V = 32768;
 constexpr int OFF_PT = NST * STAGE_BYTES;          // P~, 8 KB
-constexpr int OFF_RECV = OFF_PT + 8192;            // partial outputs from the peer: 2 x [128 d_v][32 tokens] fp32
-constexpr int RECV_BYTES = 16384;
-constexpr int SMEM_TILES = OFF_RECV + 2 * RECV_BYTES;
+constexpr int OFF_RECV = OFF_PT + 8192;            // partial outputs from the peer: 4 x [128 d_v][32 tokens] bf16
+constexpr int RECV_BYTES = 8192, NRECV = 4;
+constexpr int SMEM_TILES = OFF_RECV + NRECV * RECV_BYTES;
 constexpr int SMEM_DYN = SMEM_TILES + 1024;        // + alignment slack
 constexpr int NGA = 4, NGB = 2;                    // depth of the two rings of gate-derived factors
 // TMEM columns
 constexpr uint32_t COL_S = 0;       // fp32 state S^T, 128 columns (d_k)
 constexpr uint32_t COL_SB = 128;    // bf16 copy, 64 columns
-constexpr uint32_t COL_OA = 192;    // readout, contraction over d_k 0..63   (64 columns = tokens)
-constexpr uint32_t COL_OB = 256;    // readout, contraction over d_k 64..127 (two accumulators: two shorter MMA chains)
+constexpr uint32_t COL_O = 192;     // readout O^T, 2 x 64 columns (tokens): chunks of even / odd index
 constexpr uint32_t COL_OI = 320;    // chunk-local output O_in^T
 constexpr uint32_t COL_P = 384;     // scores P (lanes 0..63 meaningful)
 constexpr uint32_t COL_VT = 448;    // scaled V^T, bf16, 2 x 32 columns
@@ -75,9 +75,9 @@ struct alignas(16) Shared {
     uint64_t ld_full[NST], ld_empty[NST];
     uint64_t ga_full[NGA], ga_empty[NGA], gb_full[NGB], gb_empty[NGB];
     uint64_t vt_ready[2], vt_free[2];
-    uint64_t s_ready, sb_ready, u_full, o_full, o_free;
-    uint64_t p_full, p_free, pt_ready, pt_free, oi_full, oi_free;
-    uint64_t x_full[2][4];
+    uint64_t s_ready, sb_ready, u_full, o_full[2], o_free[2];
+    uint64_t p_full, pt_ready, pt_free, oi_full, oi_free;
+    uint64_t x_full[NRECV][4];
     uint32_t tmem_base;
     int abort_flag;
     GateA ga[NGA];
@@ -124,15 +124,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch behind this grid (the decode step) may be scheduled early
 
     if (tid == 0) {
-        for (int i = 0; i < NST; ++i) { mbar_init(&sh.ld_full[i], 1); mbar_init(&sh.ld_empty[i], 6); }   // two issuers + four V~ warps
+        for (int i = 0; i < NST; ++i) { mbar_init(&sh.ld_full[i], 1); mbar_init(&sh.ld_empty[i], 7); }   // three issuers + four V~ warps
         for (int i = 0; i < NGA; ++i) { mbar_init(&sh.ga_full[i], 1); mbar_init(&sh.ga_empty[i], 12); }  // eight state + four output warps
         for (int i = 0; i < NGB; ++i) { mbar_init(&sh.gb_full[i], 1); mbar_init(&sh.gb_empty[i], 4); }
         for (int i = 0; i < 2; ++i) { mbar_init(&sh.vt_ready[i], 4); mbar_init(&sh.vt_free[i], 1); }
         mbar_init(&sh.s_ready, 8); mbar_init(&sh.sb_ready, 8); mbar_init(&sh.u_full, 1);
-        mbar_init(&sh.o_full, 1); mbar_init(&sh.o_free, 4);
-        mbar_init(&sh.p_full, 1); mbar_init(&sh.p_free, 4); mbar_init(&sh.pt_ready, 4); mbar_init(&sh.pt_free, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_free[i], 4); }
+        mbar_init(&sh.p_full, 1); mbar_init(&sh.pt_ready, 4); mbar_init(&sh.pt_free, 1);
         mbar_init(&sh.oi_full, 1); mbar_init(&sh.oi_free, 4);
-        for (int b = 0; b < 2; ++b)
+        for (int b = 0; b < NRECV; ++b)
             for (int q = 0; q < 4; ++q) mbar_init(&sh.x_full[b][q], 1);
         sh.abort_flag = 0;
         fence_barrier_init();
@@ -146,15 +146,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     volatile int* abortp = &sh.abort_flag;
 #define WAIT(bar, ph) mbar_wait(bar, (uint32_t)(ph), abortp, p.status)
 
+    // Three threads issue the MMAs: a tcgen05 instruction costs its issuing thread some eighty cycles whatever its size, so
+    // the small MMAs of this kernel are issue-bound per thread, and each thread drives one dependency chain.
     if (warp == WARP_X) {
-        // ------------------------------------------------------------------ TMA producer; state update and scores
+        // ------------------------------------------------------------------ TMA producer; state update
         if (lane == 0) {
             prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
             const uint32_t sa = smem_u32(tiles);
-            constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);     // P = Q K^T: both operands K-major
             constexpr uint32_t ID_D = idesc_bf16(128, 128, 0, 1);    // S^T += V~^T K: A in TMEM, B = K as an MN-major N operand
             constexpr uint64_t ST_STEP = (uint64_t)(STAGE_BYTES >> 4);
-            const uint64_t dk_k = smem_desc_sw128(sa, 16, 1024), dq_k = smem_desc_sw128(sa + ST_Q, 16, 1024);
             const uint64_t dk_n = smem_desc_sw128(sa, 8192, 1024);
             auto load = [&](int c) {
                 const int s = c % NST;
@@ -170,69 +170,68 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     else tma_prefetch_4d(&map_v, 0, t3, 0, h);
                 }
             };
-            auto scores = [&](int c) {      // P = Q K^T of chunk c (this CTA computes its local part)
-                const int s = c % NST, n2 = c >> 1;
-                WAIT(&sh.ld_full[s], (c / NST) & 1);
-                if (n2 >= 1) WAIT(&sh.p_free, (n2 - 1) & 1);
-                tc_fence_after();
-                const uint64_t sn = (uint64_t)s * ST_STEP;
-#pragma unroll
-                for (int blk = 0; blk < 2; ++blk) {
-                    const uint64_t a = dq_k + sn + (uint64_t)(512 * blk), b = dk_k + sn + (uint64_t)(512 * blk);
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_P, a + (uint64_t)(2 * kk), b + (uint64_t)(2 * kk), ID_P, (blk | kk) ? 1u : 0u);
-                }
-                tc_commit(&sh.p_full);
-            };
             for (int c = 0; c < NST && c < nc; ++c) load(c);
 #pragma unroll 1
-            for (int c = -1; c < nc; ++c) {        // iteration -1 only issues the scores of chunk 0
-                if (c >= 0) {
-                    const int s = c % NST, b = c & 1;
-                    if (c >= 1 && c + 2 < nc) {      // the stage of chunk c - 1 takes chunk c + 2
-                        WAIT(&sh.ld_empty[(c - 1) % NST], ((c - 1) / NST) & 1);
-                        load(c + 2);
-                    }
-                    WAIT(&sh.ld_full[s], (c / NST) & 1);
-                    WAIT(&sh.vt_ready[b], (c >> 1) & 1);
-                    WAIT(&sh.s_ready, c & 1);
-                    tc_fence_after();
-                    const uint64_t bk = dk_n + (uint64_t)s * ST_STEP;
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_S, tb + COL_VT + 32 * b + 8 * kk, bk + (uint64_t)(kk * 128), ID_D, 1);
-                    tc_commit(&sh.u_full);
-                    tc_commit(&sh.vt_free[b]);
-                    tc_commit(&sh.ld_empty[s]);
+            for (int c = 0; c < nc; ++c) {
+                const int s = c % NST, b = c & 1;
+                if (c >= 1 && c + 2 < nc) {      // the stage of chunk c - 1 takes chunk c + 2
+                    WAIT(&sh.ld_empty[(c - 1) % NST], ((c - 1) / NST) & 1);
+                    load(c + 2);
                 }
-                if (c + 1 < nc && ((c + 1) & 1) == rank) scores(c + 1);
+                WAIT(&sh.ld_full[s], (c / NST) & 1);
+                WAIT(&sh.vt_ready[b], (c >> 1) & 1);
+                WAIT(&sh.s_ready, c & 1);
+                tc_fence_after();
+                const uint64_t bk = dk_n + (uint64_t)s * ST_STEP;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_ts(tb + COL_S, tb + COL_VT + 32 * b + 8 * kk, bk + (uint64_t)(kk * 128), ID_D, 1);
+                tc_commit(&sh.u_full);
+                tc_commit(&sh.vt_free[b]);
+                tc_commit(&sh.ld_empty[s]);
             }
         }
     } else if (warp == WARP_Y) {
-        // ------------------------------------------------------------------ readout and chunk-local output
+        // ------------------------------------------------------------------ readout
         if (lane == 0) {
             const uint32_t sa = smem_u32(tiles);
             constexpr uint32_t ID_C = idesc_bf16(128, 64, 0, 0);     // O^T = S^T Q^T: A in TMEM, B = Q K-major
-            constexpr uint32_t ID_B = idesc_bf16(128, 64, 1, 0);     // O_in^T = V^T P~^T: A = V as an MN-major operand
             constexpr uint64_t ST_STEP = (uint64_t)(STAGE_BYTES >> 4);
             const uint64_t dq_k = smem_desc_sw128(sa + ST_Q, 16, 1024);
-            const uint64_t dv_m = smem_desc_sw128(sa + ST_V, 8192, 1024);
-            const uint64_t dpt = smem_desc_sw128(sa + OFF_PT, 16, 1024);
 #pragma unroll 1
             for (int c = 0; c < nc; ++c) {
                 const int s = c % NST;
                 WAIT(&sh.ld_full[s], (c / NST) & 1);
-                if (c >= 1) WAIT(&sh.o_free, (c - 1) & 1);
+                if (c >= 2) WAIT(&sh.o_free[c & 1], ((c >> 1) - 1) & 1);     // the outputs of chunk c - 2 have left this accumulator
                 WAIT(&sh.sb_ready, c & 1);
                 tc_fence_after();
                 const uint64_t bq = dq_k + (uint64_t)s * ST_STEP;
+                const uint32_t od = tb + COL_O + 64 * (c & 1);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    mma_ts(tb + COL_OA, tb + COL_SB + 8 * kk, bq + (uint64_t)(2 * kk), ID_C, kk ? 1u : 0u);
-                    mma_ts(tb + COL_OB, tb + COL_SB + 32 + 8 * kk, bq + 512 + (uint64_t)(2 * kk), ID_C, kk ? 1u : 0u);
-                }
-                tc_commit(&sh.o_full);
-                if ((c & 1) == rank) {
-                    const int n2 = c >> 1;
+                for (int kk = 0; kk < 4; ++kk) mma_ts(od, tb + COL_SB + 8 * kk, bq + (uint64_t)(2 * kk), ID_C, kk ? 1u : 0u);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) mma_ts(od, tb + COL_SB + 32 + 8 * kk, bq + 512 + (uint64_t)(2 * kk), ID_C, 1u);
+                tc_commit(&sh.o_full[c & 1]);
+                tc_commit(&sh.ld_empty[s]);
+            }
+        }
+    } else if (warp == WARP_Z) {
+        // ------------------------------------------------------------------ chunk-local part: scores and O_in of the chunks this CTA owns
+        if (lane == 0) {
+            const uint32_t sa = smem_u32(tiles);
+            constexpr uint32_t ID_P = idesc_bf16(128, 64, 0, 0);     // P = Q K^T: both operands K-major
+            constexpr uint32_t ID_B = idesc_bf16(128, 64, 1, 0);     // O_in^T = V^T P~^T: A = V as an MN-major operand
+            constexpr uint64_t ST_STEP = (uint64_t)(STAGE_BYTES >> 4);
+            const uint64_t dk_k = smem_desc_sw128(sa, 16, 1024), dq_k = smem_desc_sw128(sa + ST_Q, 16, 1024);
+            const uint64_t dv_m = smem_desc_sw128(sa + ST_V, 8192, 1024);
+            const uint64_t dpt = smem_desc_sw128(sa + OFF_PT, 16, 1024);
+            // step n2 = -1 issues the scores of the first owned chunk; step n2 issues O_in of owned chunk n2 and the scores of the
+            // next one, so the decay-mask work on chunk n2 + 1 runs while the outputs of chunk n2 are finished.  In between it
+            // releases the stages of the chunks it does not touch (a commit with nothing pending arrives at once).
+#pragma unroll 1
+            for (int c = rank - 2; c < nc; c += 2) {
+                const int n2 = c >> 1;       // index of owned chunk c (c >= 0)
+                if (c >= 0) {
+                    const int s = c % NST;
                     WAIT(&sh.pt_ready, n2 & 1);
                     if (n2 >= 1) WAIT(&sh.oi_free, (n2 - 1) & 1);
                     tc_fence_after();
@@ -241,8 +240,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_OI, av + (uint64_t)(kk * 128), dpt + (uint64_t)(2 * kk), ID_B, kk ? 1u : 0u);
                     tc_commit(&sh.oi_full);
                     tc_commit(&sh.pt_free);
+                    tc_commit(&sh.ld_empty[s]);
                 }
-                tc_commit(&sh.ld_empty[s]);
+                if (c + 1 >= 0 && c + 1 < nc) {
+                    // chunk c + 1 belongs to the peer CTA: release its stage, but only once the stage holds that chunk (an arrival
+                    // before the refill would count for the stage's previous use)
+                    WAIT(&sh.ld_full[(c + 1) % NST], ((c + 1) / NST) & 1);
+                    tc_commit(&sh.ld_empty[(c + 1) % NST]);
+                }
+                if (c + 2 < nc) {
+                    const int cn = c + 2, s = cn % NST;
+                    WAIT(&sh.ld_full[s], (cn / NST) & 1);
+                    // P is free: every tile warp arrived on pt_ready for the previous owned chunk after its last read of P
+                    tc_fence_after();
+                    const uint64_t sn = (uint64_t)s * ST_STEP;
+#pragma unroll
+                    for (int blk = 0; blk < 2; ++blk) {
+                        const uint64_t a = dq_k + sn + (uint64_t)(512 * blk), b = dk_k + sn + (uint64_t)(512 * blk);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) mma_ss(tb + COL_P, a + (uint64_t)(2 * kk), b + (uint64_t)(2 * kk), ID_P, (blk | kk) ? 1u : 0u);
+                    }
+                    tc_commit(&sh.p_full);
+                }
             }
         }
     } else if (warp == WARP_GATE) {
@@ -310,7 +329,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
         }
     } else if (warp < STATE_W0) {
-        if (warp != 7) {
+        {
             // ------------------------------------------------------------------ score tile warps 0, 1, 4, 5
             // P~ rows 32 q .. 32 q + 31, columns 32 half .. 32 half + 31 of the chunks whose local part this CTA computes
             const int q = warp & 3, half = warp >> 2;
@@ -353,8 +372,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     }
                     *reinterpret_cast<uint4*>(pt + sw128_offset(j, col0)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
-                __syncwarp();
-                if (lane == 0) { tc_fence_before(); mbar_arrive(&sh.p_free); }
+                tc_fence_before();
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive(&sh.pt_ready); mbar_arrive(&sh.gb_empty[n2 & (NGB - 1)]); }
@@ -388,7 +406,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 continue;
             }
             WAIT(&sh.u_full, (c - 1) & 1);      // the update of chunk c - 1 is in the fp32 state
-            WAIT(&sh.o_full, (c - 1) & 1);      // the readout of chunk c - 1 has read the previous bf16 copy
+            WAIT(&sh.o_full[(c - 1) & 1], ((c - 1) >> 1) & 1);      // the readout of chunk c - 1 has read the previous bf16 copy
             tc_fence_after();
             const float2 a2 = make_float2(a, a);
 #pragma unroll 1
@@ -416,40 +434,45 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         tc_fence_after();
         if (g == sq.last_seg) store_state(slot_i, v, lane_addr + COL_S, 2 * ch, 2 * ch + 2);
     } else {
-        // ------------------------------------------------------------------ V~ and output warps 16..19
-        const int q = warp & 3;
+        // ------------------------------------------------------------------ V~ and output warps 16..23
+        // Two sets of four warps: set e (warps 16 + 4 e ..) takes the chunks with c mod 2 = e, so a set has two chunk periods for
+        // one chunk's work and the latencies of its steps stay off the chunk loop's critical path.
+        const int q = warp & 3, set = (warp - VE_W0) >> 2;
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
         const int v = 32 * q + lane;
-        // V~^T[v][s] = w_s V[s][v] for the update: this thread's d_v column of the V tile (two-byte loads; a warp reads 64
-        // contiguous bytes of one 128-byte row, the swizzle only permutes 16-byte pieces inside the row), two tokens per
-        // register, times the bf16 weights, into TMEM as the A operand.
-        const uint32_t vcol = (uint32_t)(v >> 6) * 8192u + (uint32_t)((v & 7) << 1);
-        const uint32_t vchunk = (uint32_t)((v & 63) >> 3);
-        const uint32_t vrow = smem_u32(tiles + ST_V) + vcol;     // + stage offset + token * 128 + (swizzled 16-byte piece)
+        // V~^T[v][s] = w_s V[s][v] for the update, into TMEM as the A operand (d_v on the lanes, two tokens per 32-bit column).
+        // ldmatrix with .trans hands a thread two consecutive tokens of one d_v column per register, which is the element
+        // pair of the operand; a 16x128b TMEM store takes exactly that distribution (lane = t / 4, column = t % 4), so the
+        // transpose costs no shuffles.  One round = 16 tokens x 16 d_v lanes: matrices (tokens 0..7 | 8..15) x (d_v 0..7 | 8..15).
+        const int mk = lane >> 3, mr = lane & 7;                 // this thread addresses row mr of matrix mk
         auto make_vt = [&](int c) {
             const int s = c % NST, b = c & 1;
             WAIT(&sh.ld_full[s], (c / NST) & 1);
             WAIT(&sh.ga_full[c & (NGA - 1)], (c / NGA) & 1);
             if (c >= 2) WAIT(&sh.vt_free[b], ((c >> 1) - 1) & 1);  // the update of chunk c - 2 has read this buffer
             tc_fence_after();
-            const uint32_t vb = vrow + (uint32_t)(s * STAGE_BYTES);
-            const uint4* wq = reinterpret_cast<const uint4*>(sh.ga[c & (NGA - 1)].w);
-            const uint32_t vt = lane_addr + COL_VT + 32 * b;
+            const uint32_t vtile = smem_u32(tiles + s * STAGE_BYTES + ST_V);
+            const uint8_t* wp = reinterpret_cast<const uint8_t*>(sh.ga[c & (NGA - 1)].w) + 4 * (lane & 3);
 #pragma unroll 1
-            for (int m = 0; m < 8; ++m) {          // eight tokens per round, loop kept rolled
-                const uint4 w4 = wq[m];
-                const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-                uint32_t raw[8];
-#pragma unroll
-                for (int r = 0; r < 8; ++r) raw[r] = ld_shared_u16(vb + (uint32_t)(m * 1024 + r * 128) + ((vchunk ^ (uint32_t)r) << 4));
-                uint32_t pk[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const uint32_t x = raw[2 * e] | (raw[2 * e + 1] << 16);
-                    const __nv_bfloat162 r2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&x), *reinterpret_cast<const __nv_bfloat162*>(&ww[e]));
-                    pk[e] = *reinterpret_cast<const uint32_t*>(&r2);
+            for (int hh = 0; hh < 2; ++hh) {       // the two 16-lane halves of this warp's TMEM quadrant
+                const int d = 32 * q + 16 * hh + 8 * (mk & 1);            // first d_v column of the matrix this thread addresses
+                // row of the V tile: token * 128 bytes, 16-byte piece (d / 8 mod 8) ^ (token mod 8); token mod 8 = mr in every round
+                const uint32_t row0 = vtile + (uint32_t)(d >> 6) * 8192u + (uint32_t)((8 * (mk >> 1) + mr) * 128) +
+                                      (((uint32_t)((d & 63) >> 3) ^ (uint32_t)mr) << 4);
+                const uint32_t vt = tb + ((uint32_t)(32 * q + 16 * hh) << 16) + COL_VT + 32 * b;
+#pragma unroll 1
+                for (int t16 = 0; t16 < 4; ++t16) {
+                    uint32_t r0, r1, r2, r3;
+                    ldmatrix_x4_trans(row0 + (uint32_t)(t16 * 16 * 128), r0, r1, r2, r3);
+                    const uint32_t w0 = *reinterpret_cast<const uint32_t*>(wp + 32 * t16), w1 = *reinterpret_cast<const uint32_t*>(wp + 32 * t16 + 16);
+                    const __nv_bfloat162 ww0 = *reinterpret_cast<const __nv_bfloat162*>(&w0), ww1 = *reinterpret_cast<const __nv_bfloat162*>(&w1);
+                    __nv_bfloat162 y0 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r0), ww0);
+                    __nv_bfloat162 y1 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r1), ww0);
+                    __nv_bfloat162 y2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r2), ww1);
+                    __nv_bfloat162 y3 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r3), ww1);
+                    tmem_st_16x128b(vt + 8 * t16, *reinterpret_cast<const uint32_t*>(&y0), *reinterpret_cast<const uint32_t*>(&y1));
+                    tmem_st_16x128b(vt + 8 * t16 + 4, *reinterpret_cast<const uint32_t*>(&y2), *reinterpret_cast<const uint32_t*>(&y3));
                 }
-                tmem_st4(vt + 4 * m, pk);
             }
             tc_wait_st();
             tc_fence_before();
@@ -457,24 +480,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (lane == 0) { mbar_arrive(&sh.vt_ready[b]); mbar_arrive(&sh.ld_empty[s]); }
         };
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
-        const uint32_t recv_row = (uint32_t)v * 128u;                        // this thread's row in a receive buffer
+        // receive buffers: [128 d_v rows][32 tokens] bf16, 64-byte rows; 16-byte piece k of row v sits at piece k ^ ((v >> 1) & 3)
+        const uint32_t recv_row = (uint32_t)v * 64u, vsw = (uint32_t)((v >> 1) & 3);
         const uint32_t recv_peer = map_to_cta(smem_u32(tiles + OFF_RECV), (uint32_t)peer) + recv_row;
-        const uint32_t xfull_peer0 = map_to_cta(smem_u32(&sh.x_full[0][q]), (uint32_t)peer);
-        const uint32_t xfull_peer1 = map_to_cta(smem_u32(&sh.x_full[1][q]), (uint32_t)peer);
-        const uint32_t vsw = (uint32_t)(v & 7);
-        // Partial outputs of 16 tokens (columns col .. col + 15 of the accumulators) of chunk c for this thread's d_v lane:
-        // rowf_j (O_a + O_b) [+ O_in]
+        const uint32_t xfull_peer = map_to_cta(smem_u32(&sh.x_full[0][q]), (uint32_t)peer);     // + 32 bytes per buffer index
+        // Partial outputs of 16 tokens (columns col .. col + 15 of the accumulator) of chunk c for this thread's d_v lane:
+        // rowf_j O^i[j] [+ O_in[j]]
         auto partial16 = [&](int c, int col, float (&x)[16]) {
-            uint32_t ra[16], rb[16];
-            tmem_ld16(lane_addr + COL_OA + col, ra);
-            tmem_ld16(lane_addr + COL_OB + col, rb);
+            uint32_t ra[16];
+            tmem_ld16(lane_addr + COL_O + 64 * (c & 1) + col, ra);
             const float4* rf = reinterpret_cast<const float4*>(sh.ga[c & (NGA - 1)].rowf + col);
             float f[16];
 #pragma unroll
             for (int m = 0; m < 4; ++m) { const float4 t = rf[m]; f[4 * m] = t.x; f[4 * m + 1] = t.y; f[4 * m + 2] = t.z; f[4 * m + 3] = t.w; }
             tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 16; ++k) x[k] = f[k] * (__uint_as_float(ra[k]) + __uint_as_float(rb[k]));
+            for (int k = 0; k < 16; ++k) x[k] = f[k] * __uint_as_float(ra[k]);
             if ((c & 1) == rank) {
                 tmem_ld16(lane_addr + COL_OI + col, ra);
                 tc_wait_ld();
@@ -482,30 +503,32 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 for (int k = 0; k < 16; ++k) x[k] += __uint_as_float(ra[k]);
             }
         };
+        if (set < nc) make_vt(set);
 #pragma unroll 1
-        for (int c = -1; c < nc; ++c) {       // iteration -1 only prepares chunk 0
-            if (c + 1 < nc) make_vt(c + 1);
-            if (c < 0) continue;
-            const int b = c & 1;
-            WAIT(&sh.o_full, c & 1);
+        for (int c = set; c < nc; c += 2) {
+            const int b = c & (NRECV - 1);
+            WAIT(&sh.o_full[c & 1], (c >> 1) & 1);
             if ((c & 1) == rank) WAIT(&sh.oi_full, (c >> 1) & 1);
             tc_fence_after();
-            // ---- the peer's 32 tokens: send.  Its receive buffer b is free: the peer read what chunk c - 2 left there before it
-            // sent its part of chunk c - 1, which this warp has waited for.  The stores complete on the peer's barrier.
+            // ---- the peer's 32 tokens: send (bf16).  The peer's receive buffer b is free: the peer's warp read what chunk c - 4
+            // left there before it sent its part of chunk c - 2, which this warp has waited for.  The stores complete on the
+            // peer's barrier.
             {
-                const uint32_t dst = recv_peer + (uint32_t)b * RECV_BYTES, bar = b ? xfull_peer1 : xfull_peer0;
+                const uint32_t dst = recv_peer + (uint32_t)b * RECV_BYTES, bar = xfull_peer + (uint32_t)b * 32u;
 #pragma unroll 1
                 for (int i = 0; i < 2; ++i) {
                     float x[16];
                     partial16(c, 32 * peer + 16 * i, x);
+                    uint32_t pk[8];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        st_async_f32x4(dst + (((uint32_t)(4 * i + k) ^ vsw) << 4), x[4 * k], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3], bar);
+                    for (int k = 0; k < 8; ++k) pk[k] = pack_bf16(x[2 * k], x[2 * k + 1]);
+                    st_async_b32x4(dst + (((uint32_t)(2 * i) ^ vsw) << 4), pk[0], pk[1], pk[2], pk[3], bar);
+                    st_async_b32x4(dst + (((uint32_t)(2 * i + 1) ^ vsw) << 4), pk[4], pk[5], pk[6], pk[7], bar);
                 }
             }
             // ---- own 32 tokens: add what the peer sent, store
-            if (lane == 0) mbar_arrive_expect_tx(&sh.x_full[b][q], 32 * 128);      // the peer's warp q sends 128 bytes per lane
-            mbar_wait_cluster(&sh.x_full[b][q], (uint32_t)((c >> 1) & 1), abortp, p.status);
+            if (lane == 0) mbar_arrive_expect_tx(&sh.x_full[b][q], 32 * 64);      // the peer's warp q sends 64 bytes per lane
+            mbar_wait_cluster(&sh.x_full[b][q], (uint32_t)((c >> 2) & 1), abortp, p.status);
             {
                 const int valid = min(C, sq.len - tok0 - c * C) - 32 * rank;     // tokens of this CTA's half that exist
                 // a thread owns one d_v lane; a warp's store of one token is 64 contiguous bytes (two full sectors)
@@ -517,9 +540,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     float x[16];
                     partial16(c, 32 * rank + 16 * i, x);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float4 y = *reinterpret_cast<const float4*>(src + (((uint32_t)(4 * i + k) ^ vsw) << 4));
-                        x[4 * k] += y.x; x[4 * k + 1] += y.y; x[4 * k + 2] += y.z; x[4 * k + 3] += y.w;
+                    for (int k = 0; k < 2; ++k) {
+                        const uint4 y = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * i + k) ^ vsw) << 4));
+                        const uint32_t yy[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            x[8 * k + 2 * e] += __uint_as_float(yy[e] << 16);
+                            x[8 * k + 2 * e + 1] += __uint_as_float(yy[e] & 0xffff0000u);
+                        }
                     }
                     if (valid >= 16 * i + 16) {
 #pragma unroll
@@ -534,10 +562,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             __syncwarp();
             if (lane == 0) {
                 tc_fence_before();
-                mbar_arrive(&sh.o_free);
+                mbar_arrive(&sh.o_free[c & 1]);
                 if ((c & 1) == rank) mbar_arrive(&sh.oi_free);
                 mbar_arrive(&sh.ga_empty[c & (NGA - 1)]);
             }
+            if (c + 2 < nc) make_vt(c + 2);
         }
     }
 #undef WAIT

@@ -21,16 +21,15 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// (waits poll with mbarrier.test_wait: mbarrier.try_wait would park the thread for a while before it reports "not yet")
 
 // Bounded wait.  The fast path (phase already complete) is a single inlined test; otherwise a
-// non-inlined loop polls with a short sleep between tests.  It gives up after `limit` polls, raises
-// *abort_flag (shared) and *status (global) and returns false.  Once the abort flag is up every
+// non-inlined loop parks the thread on the barrier (mbarrier.try_wait) again and again.  It gives up
+// after `limit` rounds or about a second, raises *abort_flag (shared) and *status (global) and returns false.  Once the abort flag is up every
 // later wait returns on its first poll, so a CTA that lost a signal still runs to its end, frees its
 // TMEM and exits instead of hanging.  CLUSTER = true makes the successful test an acquire at
 // cluster scope (data another CTA of the cluster wrote into this CTA's shared memory before its
 // remote arrive is then visible).
-constexpr uint32_t MBAR_WAIT_LIMIT = 4000000u;   // polls of a hundred nanoseconds or more each: about a second
+constexpr uint32_t MBAR_WAIT_LIMIT = 0x7fffffffu;   // parked waits; the one-second clock check ends a lost wait long before
 
 template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_test_wait_t(uint64_t* bar, uint32_t parity) {
@@ -49,13 +48,38 @@ __device__ __forceinline__ bool mbar_test_wait_t(uint64_t* bar, uint32_t parity)
             : "memory");
     return ok != 0;
 }
+// One parked wait: the hardware suspends the thread until the phase completes or about a microsecond has passed, so a
+// waiter wakes as soon as the barrier flips and executes no polling instructions meanwhile.
+template <bool CLUSTER>
+__device__ __forceinline__ bool mbar_try_wait_t(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    if (CLUSTER)
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
+            : "memory");
+    else
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
+            : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Gives up after `limit` parked waits or about a second, whichever comes first.
 template <bool CLUSTER>
 __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, uint32_t limit) {
+    const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0; i < limit; ++i) {
-        if (mbar_test_wait_t<CLUSTER>(bar, parity)) return true;
-        if ((i & 63u) == 0u && *abort_flag) return false;
-        __nanosleep(100);  // a hot spin takes issue slots from the warps that are doing the work (measured: +4 % run time);
-                           // sleeps of 20..400 ns are equal within noise, 1 us costs 10 %
+        if (mbar_try_wait_t<CLUSTER>(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if ((i & 15u) == 15u && global_timer_ns() - t0 > 1000000000ull) break;
     }
     *abort_flag = 1;
     atomicExch(status, 5 /* DSLA_ERR_TIMEOUT */);
@@ -103,6 +127,11 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr) {
 __device__ __forceinline__ void st_async_f32x4(uint32_t caddr, float a, float b, float c, float d, uint32_t cbar) {
     asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(caddr), "f"(a), "f"(b),
                  "f"(c), "f"(d), "r"(cbar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_b32x4(uint32_t caddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t cbar) {
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(caddr), "r"(a), "r"(b),
+                 "r"(c), "r"(d), "r"(cbar)
                  : "memory");
 }
 // Arrive on an mbarrier of another CTA without ordering anything (a "buffer is free" signal after its reads returned).
@@ -216,6 +245,19 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&v)[8]) {
 }
 __device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint32_t (&v)[4]) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%4], {%0,%1,%2,%3};" ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(taddr)
+                 : "memory");
+}
+// 16 lanes x 128 bits (four 32-bit columns): thread t of the warp supplies column t % 4 of lane t / 4 (a) and of
+// lane t / 4 + 8 (b) -- the layout in which ldmatrix hands out 8x8 matrices of 16-bit elements.
+__device__ __forceinline__ void tmem_st_16x128b(uint32_t taddr, uint32_t a, uint32_t b) {
+    asm volatile("tcgen05.st.sync.aligned.16x128b.x1.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(a), "r"(b) : "memory");
+}
+// Four 8x8 matrices of 16-bit elements, transposed: thread t supplies the address of row t % 8 of matrix t / 8 and
+// receives, per matrix, the elements (rows 2 (t % 4), 2 (t % 4) + 1; column t / 4) in the low / high half of a register.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t saddr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(saddr)
                  : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
