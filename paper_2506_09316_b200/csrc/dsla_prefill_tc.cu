@@ -48,7 +48,9 @@ constexpr int STAGE_BYTES = 3 * 16384, ST_Q = 16384, ST_V = 32768;
 constexpr int OFF_PT = NST * STAGE_BYTES;          // P~, 8 KB
 constexpr int OFF_RECV = OFF_PT + 8192;            // partial outputs from the peer: 4 x [128 d_v][32 tokens] bf16
 constexpr int RECV_BYTES = 8192, NRECV = 4;
-constexpr int SMEM_TILES = OFF_RECV + NRECV * RECV_BYTES;
+constexpr int OFF_OUT = OFF_RECV + NRECV * RECV_BYTES;      // finished outputs, token-major: per finishing warp [32 tokens][32 d_v] bf16
+constexpr int OUT_PITCH = 80, OUT_WARP_BYTES = 32 * OUT_PITCH;    // 64-byte rows padded to 80 (stmatrix rows hit distinct banks)
+constexpr int SMEM_TILES = OFF_OUT + 4 * OUT_WARP_BYTES;
 constexpr int SMEM_DYN = SMEM_TILES + 1024;        // + alignment slack
 constexpr int NGA = 4, NGB = 2;                    // depth of the two rings of gate-derived factors
 // TMEM columns
@@ -77,7 +79,7 @@ struct alignas(16) Shared {
     uint64_t vt_ready[2], vt_free[2];
     uint64_t s_ready, sb_ready, u_full, o_full[2], o_free[2];
     uint64_t p_full, pt_ready, pt_free, oi_full, oi_free;
-    uint64_t x_full[NRECV][4];
+    uint64_t x_full[NRECV][4], x_free[NRECV][4];
     uint32_t tmem_base;
     int abort_flag;
     GateA ga[NGA];
@@ -125,15 +127,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
     if (tid == 0) {
         for (int i = 0; i < NST; ++i) { mbar_init(&sh.ld_full[i], 1); mbar_init(&sh.ld_empty[i], 7); }   // three issuers + four V~ warps
-        for (int i = 0; i < NGA; ++i) { mbar_init(&sh.ga_full[i], 1); mbar_init(&sh.ga_empty[i], 12); }  // eight state + four output warps
+        for (int i = 0; i < NGA; ++i) { mbar_init(&sh.ga_full[i], 1); mbar_init(&sh.ga_empty[i], 16); }  // eight state + eight output warps
         for (int i = 0; i < NGB; ++i) { mbar_init(&sh.gb_full[i], 1); mbar_init(&sh.gb_empty[i], 4); }
         for (int i = 0; i < 2; ++i) { mbar_init(&sh.vt_ready[i], 4); mbar_init(&sh.vt_free[i], 1); }
         mbar_init(&sh.s_ready, 8); mbar_init(&sh.sb_ready, 8); mbar_init(&sh.u_full, 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_free[i], 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh.o_full[i], 1); mbar_init(&sh.o_free[i], 8); }
         mbar_init(&sh.p_full, 1); mbar_init(&sh.pt_ready, 4); mbar_init(&sh.pt_free, 1);
-        mbar_init(&sh.oi_full, 1); mbar_init(&sh.oi_free, 4);
+        mbar_init(&sh.oi_full, 1); mbar_init(&sh.oi_free, 8);
         for (int b = 0; b < NRECV; ++b)
-            for (int q = 0; q < 4; ++q) mbar_init(&sh.x_full[b][q], 1);
+            for (int q = 0; q < 4; ++q) { mbar_init(&sh.x_full[b][q], 1); mbar_init(&sh.x_free[b][q], 1); }
         sh.abort_flag = 0;
         fence_barrier_init();
     }
@@ -435,8 +437,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (g == sq.last_seg) store_state(slot_i, v, lane_addr + COL_S, 2 * ch, 2 * ch + 2);
     } else {
         // ------------------------------------------------------------------ V~ and output warps 16..23
-        // Two sets of four warps: set e (warps 16 + 4 e ..) takes the chunks with c mod 2 = e, so a set has two chunk periods for
-        // one chunk's work and the latencies of its steps stay off the chunk loop's critical path.
+        // Two sets of four warps: warps 16..19 prepare V~ and send the peer CTA its half of every chunk's outputs, warps 20..23
+        // finish this CTA's half; both read the same accumulators.
         const int q = warp & 3, set = (warp - VE_W0) >> 2;
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
         const int v = 32 * q + lane;
@@ -480,85 +482,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (lane == 0) { mbar_arrive(&sh.vt_ready[b]); mbar_arrive(&sh.ld_empty[s]); }
         };
         __nv_bfloat16* og = reinterpret_cast<__nv_bfloat16*>(p.o);
-        // receive buffers: [128 d_v rows][32 tokens] bf16, 64-byte rows; 16-byte piece k of row v sits at piece k ^ ((v >> 1) & 3)
-        const uint32_t recv_row = (uint32_t)v * 64u, vsw = (uint32_t)((v >> 1) & 3);
-        const uint32_t recv_peer = map_to_cta(smem_u32(tiles + OFF_RECV), (uint32_t)peer) + recv_row;
-        const uint32_t xfull_peer = map_to_cta(smem_u32(&sh.x_full[0][q]), (uint32_t)peer);     // + 32 bytes per buffer index
-        // Partial outputs of 16 tokens (columns col .. col + 15 of the accumulator) of chunk c for this thread's d_v lane:
-        // rowf_j O^i[j] [+ O_in[j]]
-        auto partial16 = [&](int c, int col, float (&x)[16]) {
+        // The accumulators are read in the 16x256b distribution: per 16-lane half hh of this warp's quadrant, thread t holds the
+        // d_v lanes 32 q + 16 hh + t / 4 (and + 8) and, per group i of 8 tokens, the token pair 8 i + 2 (t % 4), + 1.  A pair of
+        // tokens of one d_v lane packs into one bf16x2 register, the unit of the exchange with the peer CTA (slot of 16 bytes
+        // per thread, group pair and half) and of the transposing stmatrix that lays the finished outputs out token-major.
+        // x[4 i + 0, 1]: lane t / 4, x[4 i + 2, 3]: lane t / 4 + 8 ; value = rowf_j O^i[j] [+ O_in[j]]
+        const int tq = lane & 3;
+        auto partial32 = [&](int c, int hh, int th, float2 (&x)[8]) {
             uint32_t ra[16];
-            tmem_ld16(lane_addr + COL_O + 64 * (c & 1) + col, ra);
-            const float4* rf = reinterpret_cast<const float4*>(sh.ga[c & (NGA - 1)].rowf + col);
-            float f[16];
+            const uint32_t ta = tb + ((uint32_t)(32 * q + 16 * hh) << 16) + 32 * th;
+            tmem_ld_16x256b_x4(ta + COL_O + 64 * (c & 1), ra);
+            const float* rfp = sh.ga[c & (NGA - 1)].rowf + 32 * th + 2 * tq;
+            float2 f[4];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) { const float4 t = rf[m]; f[4 * m] = t.x; f[4 * m + 1] = t.y; f[4 * m + 2] = t.z; f[4 * m + 3] = t.w; }
+            for (int i = 0; i < 4; ++i) f[i] = *reinterpret_cast<const float2*>(rfp + 8 * i);
             tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 16; ++k) x[k] = f[k] * __uint_as_float(ra[k]);
+            for (int i = 0; i < 4; ++i) {
+                x[2 * i] = __fmul2_rn(make_float2(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1])), f[i]);
+                x[2 * i + 1] = __fmul2_rn(make_float2(__uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3])), f[i]);
+            }
             if ((c & 1) == rank) {
-                tmem_ld16(lane_addr + COL_OI + col, ra);
+                tmem_ld_16x256b_x4(ta + COL_OI, ra);
                 tc_wait_ld();
 #pragma unroll
-                for (int k = 0; k < 16; ++k) x[k] += __uint_as_float(ra[k]);
+                for (int i = 0; i < 8; ++i) x[i] = __fadd2_rn(x[i], make_float2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])));
             }
         };
-        if (set < nc) make_vt(set);
-#pragma unroll 1
-        for (int c = set; c < nc; c += 2) {
-            const int b = c & (NRECV - 1);
-            WAIT(&sh.o_full[c & 1], (c >> 1) & 1);
-            if ((c & 1) == rank) WAIT(&sh.oi_full, (c >> 1) & 1);
-            tc_fence_after();
-            // ---- the peer's 32 tokens: send (bf16).  The peer's receive buffer b is free: the peer's warp read what chunk c - 4
-            // left there before it sent its part of chunk c - 2, which this warp has waited for.  The stores complete on the
-            // peer's barrier.
-            {
-                const uint32_t dst = recv_peer + (uint32_t)b * RECV_BYTES, bar = xfull_peer + (uint32_t)b * 32u;
-#pragma unroll 1
-                for (int i = 0; i < 2; ++i) {
-                    float x[16];
-                    partial16(c, 32 * peer + 16 * i, x);
-                    uint32_t pk[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) pk[k] = pack_bf16(x[2 * k], x[2 * k + 1]);
-                    st_async_b32x4(dst + (((uint32_t)(2 * i) ^ vsw) << 4), pk[0], pk[1], pk[2], pk[3], bar);
-                    st_async_b32x4(dst + (((uint32_t)(2 * i + 1) ^ vsw) << 4), pk[4], pk[5], pk[6], pk[7], bar);
-                }
-            }
-            // ---- own 32 tokens: add what the peer sent, store
-            if (lane == 0) mbar_arrive_expect_tx(&sh.x_full[b][q], 32 * 64);      // the peer's warp q sends 64 bytes per lane
-            mbar_wait_cluster(&sh.x_full[b][q], (uint32_t)((c >> 2) & 1), abortp, p.status);
-            {
-                const int valid = min(C, sq.len - tok0 - c * C) - 32 * rank;     // tokens of this CTA's half that exist
-                // a thread owns one d_v lane; a warp's store of one token is 64 contiguous bytes (two full sectors)
-                __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * rank) * p.H + h) * D + v;
-                const size_t row = (size_t)p.H * D;
-                const uint8_t* src = tiles + OFF_RECV + b * RECV_BYTES + recv_row;
-#pragma unroll 1
-                for (int i = 0; i < 2; ++i) {
-                    float x[16];
-                    partial16(c, 32 * rank + 16 * i, x);
-#pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        const uint4 y = *reinterpret_cast<const uint4*>(src + (((uint32_t)(2 * i + k) ^ vsw) << 4));
-                        const uint32_t yy[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            x[8 * k + 2 * e] += __uint_as_float(yy[e] << 16);
-                            x[8 * k + 2 * e + 1] += __uint_as_float(yy[e] & 0xffff0000u);
-                        }
-                    }
-                    if (valid >= 16 * i + 16) {
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj) dst[(16 * i + jj) * row] = __float2bfloat16_rn(x[jj]);
-                    } else {
-#pragma unroll
-                        for (int jj = 0; jj < 16; ++jj)
-                            if (16 * i + jj < valid) dst[(16 * i + jj) * row] = __float2bfloat16_rn(x[jj]);
-                    }
-                }
-            }
+        auto release = [&](int c) {       // this warp has read its part of the accumulators and of the chunk's factors
             __syncwarp();
             if (lane == 0) {
                 tc_fence_before();
@@ -566,7 +517,87 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if ((c & 1) == rank) mbar_arrive(&sh.oi_free);
                 mbar_arrive(&sh.ga_empty[c & (NGA - 1)]);
             }
-            if (c + 2 < nc) make_vt(c + 2);
+        };
+        // receive buffers: per warp q 2 KB = [half hh][piece k][lane] x 16 bytes (two bf16x2 group pairs per piece)
+        const uint32_t slot = (uint32_t)(q * 2048 + lane * 16);
+        if (set == 0) {
+            // ---- sending warps: V~ one chunk ahead (it feeds the state chain), then the peer's 32 tokens of the chunk's outputs
+            // as bf16 partial sums into the peer's receive buffer; the stores complete on the peer's barrier.
+            const uint32_t recv_peer = map_to_cta(smem_u32(tiles + OFF_RECV), (uint32_t)peer) + slot;
+            const uint32_t xfull_peer = map_to_cta(smem_u32(&sh.x_full[0][q]), (uint32_t)peer);     // + 32 bytes per buffer index
+#pragma unroll 1
+            for (int c = -1; c < nc; ++c) {
+                if (c + 1 < nc) make_vt(c + 1);
+                if (c < 0) continue;
+                const int b = c & (NRECV - 1);
+                WAIT(&sh.o_full[c & 1], (c >> 1) & 1);
+                if ((c & 1) == rank) WAIT(&sh.oi_full, (c >> 1) & 1);
+                if (c >= NRECV) WAIT(&sh.x_free[b][q], ((c / NRECV) - 1) & 1);     // the peer has read what chunk c - 4 left in buffer b
+                tc_fence_after();
+                const uint32_t dst = recv_peer + (uint32_t)b * RECV_BYTES, bar = xfull_peer + (uint32_t)b * 32u;
+#pragma unroll 1
+                for (int hh = 0; hh < 2; ++hh) {
+                    float2 x[8];
+                    partial32(c, hh, peer, x);
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) pk[k] = pack_bf16(x[k].x, x[k].y);
+                    st_async_b32x4(dst + (uint32_t)(hh * 1024), pk[0], pk[1], pk[2], pk[3], bar);
+                    st_async_b32x4(dst + (uint32_t)(hh * 1024 + 512), pk[4], pk[5], pk[6], pk[7], bar);
+                }
+                release(c);
+            }
+        } else {
+            // ---- finishing warps: this CTA's 32 tokens: own partial sums + what the peer sent -> bf16 -> token-major staging tile
+            // (stmatrix, transposed) -> 16-byte stores to global memory
+            const uint32_t xfree_peer = map_to_cta(smem_u32(&sh.x_free[0][q]), (uint32_t)peer);     // + 32 bytes per buffer index
+            uint8_t* stage = tiles + OFF_OUT + q * OUT_WARP_BYTES;                 // [32 tokens][32 d_v] bf16, rows OUT_PITCH bytes apart
+            const uint32_t st_row = smem_u32(stage) + (uint32_t)((lane & 7) * OUT_PITCH + (lane >> 3) * 16);   // stmatrix: row lane % 8 of matrix lane / 8
+#pragma unroll 1
+            for (int c = 0; c < nc; ++c) {
+                const int b = c & (NRECV - 1);
+                if (lane == 0) mbar_arrive_expect_tx(&sh.x_full[b][q], 32 * 64);      // the peer's warp q sends 64 bytes per lane
+                WAIT(&sh.o_full[c & 1], (c >> 1) & 1);
+                if ((c & 1) == rank) WAIT(&sh.oi_full, (c >> 1) & 1);
+                tc_fence_after();
+                uint32_t out[2][8];          // [hh][2 i + (lane t/4 | lane t/4 + 8)] : bf16x2 of the token pair
+                float2 x[8];
+                partial32(c, 0, rank, x);
+                mbar_wait_cluster(&sh.x_full[b][q], (uint32_t)((c / NRECV) & 1), abortp, p.status);
+                const uint8_t* src = tiles + OFF_RECV + b * RECV_BYTES + slot;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    if (hh == 1) partial32(c, 1, rank, x);
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const uint4 y = *reinterpret_cast<const uint4*>(src + hh * 1024 + k * 512);
+                        const uint32_t yy[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 s2 = __fadd2_rn(x[4 * k + e], make_float2(__uint_as_float(yy[e] << 16), __uint_as_float(yy[e] & 0xffff0000u)));
+                            out[hh][4 * k + e] = pack_bf16(s2.x, s2.y);
+                        }
+                    }
+                }
+                release(c);
+                if (lane == 0) mbar_arrive_cluster_relaxed(xfree_peer + (uint32_t)b * 32u);     // after release(): the reads have returned
+                // matrices of group i: d_v blocks (hh 0: t/4, t/4 + 8; hh 1: t/4, t/4 + 8) x tokens 8 i .. 8 i + 7
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    stmatrix_x4_trans(st_row + (uint32_t)(8 * i * OUT_PITCH), out[0][2 * i], out[0][2 * i + 1], out[1][2 * i], out[1][2 * i + 1]);
+                __syncwarp();
+                const int valid = min(C, sq.len - tok0 - c * C) - 32 * rank;     // tokens of this CTA's half that exist
+                // a warp store covers 8 tokens x 64 contiguous bytes
+                __nv_bfloat16* dst = og + ((size_t)(t0 + c * C + 32 * rank) * p.H + h) * D + 32 * q + 8 * (lane & 3);
+                const size_t row = (size_t)p.H * D;
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    const int tok = (lane >> 2) + 8 * m;
+                    const uint4 y = *reinterpret_cast<const uint4*>(stage + tok * OUT_PITCH + (lane & 3) * 16);
+                    if (tok < valid) *reinterpret_cast<uint4*>(dst + tok * row) = y;
+                }
+                __syncwarp();
+            }
         }
     }
 #undef WAIT

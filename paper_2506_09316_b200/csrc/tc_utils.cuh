@@ -247,6 +247,21 @@ __device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint32_t (&v)[4])
     asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%4], {%0,%1,%2,%3};" ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(taddr)
                  : "memory");
 }
+// 16 lanes x 32 columns in the 16x256b distribution (the accumulator layout of mma fragments): for each group i of 8
+// columns, thread t receives columns 8 i + 2 (t % 4) and + 1 of lane t / 4 (v[4 i], v[4 i + 1]) and of lane t / 4 + 8
+// (v[4 i + 2], v[4 i + 3]).
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : DSLA_R8(v, 0), DSLA_R8(v, 8)
+                 : "r"(taddr)
+                 : "memory");
+}
+// Stores four 8x8 matrices of 16-bit elements transposed: thread t holds, per matrix, the elements (row t / 4, columns
+// 2 (t % 4), + 1); memory row r of matrix k (address supplied by thread 8 k + r) receives column r of that matrix.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t saddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+                 : "memory");
+}
 // 16 lanes x 128 bits (four 32-bit columns): thread t of the warp supplies column t % 4 of lane t / 4 (a) and of
 // lane t / 4 + 8 (b) -- the layout in which ldmatrix hands out 8x8 matrices of 16-bit elements.
 __device__ __forceinline__ void tmem_st_16x128b(uint32_t taddr, uint32_t a, uint32_t b) {
