@@ -176,10 +176,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll 1
             for (int c = 0; c < nc; ++c) {
                 const int s = c % NST, b = c & 1;
-                if (c >= 1 && c + 2 < nc) {      // the stage of chunk c - 1 takes chunk c + 2
-                    WAIT(&sh.ld_empty[(c - 1) % NST], ((c - 1) / NST) & 1);
-                    load(c + 2);
-                }
                 WAIT(&sh.ld_full[s], (c / NST) & 1);
                 WAIT(&sh.vt_ready[b], (c >> 1) & 1);
                 WAIT(&sh.s_ready, c & 1);
@@ -190,6 +186,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_commit(&sh.u_full);
                 tc_commit(&sh.vt_free[b]);
                 tc_commit(&sh.ld_empty[s]);
+                // after the update is on its way: the stage of chunk c - 1 takes chunk c + 2
+                if (c >= 1 && c + 2 < nc) {
+                    WAIT(&sh.ld_empty[(c - 1) % NST], ((c - 1) / NST) & 1);
+                    load(c + 2);
+                }
             }
         }
     } else if (warp == WARP_Y) {
@@ -462,16 +463,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const uint32_t row0 = vtile + (uint32_t)(d >> 6) * 8192u + (uint32_t)((8 * (mk >> 1) + mr) * 128) +
                                       (((uint32_t)((d & 63) >> 3) ^ (uint32_t)mr) << 4);
                 const uint32_t vt = tb + ((uint32_t)(32 * q + 16 * hh) << 16) + COL_VT + 32 * b;
-#pragma unroll 1
+                uint32_t r[16], w[8];
+#pragma unroll
+                for (int t16 = 0; t16 < 4; ++t16) {      // all loads of the half first: their latencies overlap
+                    ldmatrix_x4_trans(row0 + (uint32_t)(t16 * 16 * 128), r[4 * t16], r[4 * t16 + 1], r[4 * t16 + 2], r[4 * t16 + 3]);
+                    w[2 * t16] = *reinterpret_cast<const uint32_t*>(wp + 32 * t16);
+                    w[2 * t16 + 1] = *reinterpret_cast<const uint32_t*>(wp + 32 * t16 + 16);
+                }
+#pragma unroll
                 for (int t16 = 0; t16 < 4; ++t16) {
-                    uint32_t r0, r1, r2, r3;
-                    ldmatrix_x4_trans(row0 + (uint32_t)(t16 * 16 * 128), r0, r1, r2, r3);
-                    const uint32_t w0 = *reinterpret_cast<const uint32_t*>(wp + 32 * t16), w1 = *reinterpret_cast<const uint32_t*>(wp + 32 * t16 + 16);
-                    const __nv_bfloat162 ww0 = *reinterpret_cast<const __nv_bfloat162*>(&w0), ww1 = *reinterpret_cast<const __nv_bfloat162*>(&w1);
-                    __nv_bfloat162 y0 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r0), ww0);
-                    __nv_bfloat162 y1 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r1), ww0);
-                    __nv_bfloat162 y2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r2), ww1);
-                    __nv_bfloat162 y3 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r3), ww1);
+                    const __nv_bfloat162 ww0 = *reinterpret_cast<const __nv_bfloat162*>(&w[2 * t16]), ww1 = *reinterpret_cast<const __nv_bfloat162*>(&w[2 * t16 + 1]);
+                    const __nv_bfloat162 y0 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16]), ww0);
+                    const __nv_bfloat162 y1 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16 + 1]), ww0);
+                    const __nv_bfloat162 y2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16 + 2]), ww1);
+                    const __nv_bfloat162 y3 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16 + 3]), ww1);
                     tmem_st_16x128b(vt + 8 * t16, *reinterpret_cast<const uint32_t*>(&y0), *reinterpret_cast<const uint32_t*>(&y1));
                     tmem_st_16x128b(vt + 8 * t16 + 4, *reinterpret_cast<const uint32_t*>(&y2), *reinterpret_cast<const uint32_t*>(&y3));
                 }
@@ -489,24 +494,30 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // x[4 i + 0, 1]: lane t / 4, x[4 i + 2, 3]: lane t / 4 + 8 ; value = rowf_j O^i[j] [+ O_in[j]]
         const int tq = lane & 3;
         auto partial32 = [&](int c, int hh, int th, float2 (&x)[8]) {
-            uint32_t ra[16];
+            uint32_t ra[16], rc[16];
             const uint32_t ta = tb + ((uint32_t)(32 * q + 16 * hh) << 16) + 32 * th;
+            const bool own = (c & 1) == rank;       // this CTA computed the chunk-local part
             tmem_ld_16x256b_x4(ta + COL_O + 64 * (c & 1), ra);
+            if (own) tmem_ld_16x256b_x4(ta + COL_OI, rc);
             const float* rfp = sh.ga[c & (NGA - 1)].rowf + 32 * th + 2 * tq;
             float2 f[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) f[i] = *reinterpret_cast<const float2*>(rfp + 8 * i);
             tc_wait_ld();
+            if (own) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                x[2 * i] = __fmul2_rn(make_float2(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1])), f[i]);
-                x[2 * i + 1] = __fmul2_rn(make_float2(__uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3])), f[i]);
-            }
-            if ((c & 1) == rank) {
-                tmem_ld_16x256b_x4(ta + COL_OI, ra);
-                tc_wait_ld();
+                for (int i = 0; i < 4; ++i) {
+                    x[2 * i] = __ffma2_rn(make_float2(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1])), f[i],
+                                          make_float2(__uint_as_float(rc[4 * i]), __uint_as_float(rc[4 * i + 1])));
+                    x[2 * i + 1] = __ffma2_rn(make_float2(__uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3])), f[i],
+                                              make_float2(__uint_as_float(rc[4 * i + 2]), __uint_as_float(rc[4 * i + 3])));
+                }
+            } else {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) x[i] = __fadd2_rn(x[i], make_float2(__uint_as_float(ra[2 * i]), __uint_as_float(ra[2 * i + 1])));
+                for (int i = 0; i < 4; ++i) {
+                    x[2 * i] = __fmul2_rn(make_float2(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1])), f[i]);
+                    x[2 * i + 1] = __fmul2_rn(make_float2(__uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3])), f[i]);
+                }
             }
         };
         auto release = [&](int c) {       // this warp has read its part of the accumulators and of the chunk's factors

@@ -48,7 +48,7 @@ __device__ __forceinline__ bool mbar_test_wait_t(uint64_t* bar, uint32_t parity)
             : "memory");
     return ok != 0;
 }
-// One parked wait: the hardware suspends the thread until the phase completes or about a microsecond has passed, so a
+// One parked wait: the hardware suspends the thread until the phase completes or its time limit (a hint of 0.1 ms here) has passed, so a
 // waiter wakes as soon as the barrier flips and executes no polling instructions meanwhile.
 template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_try_wait_t(uint64_t* bar, uint32_t parity) {
@@ -57,13 +57,13 @@ __device__ __forceinline__ bool mbar_try_wait_t(uint64_t* bar, uint32_t parity) 
         asm volatile(
             "{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
             : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(100000u)
             : "memory");
     else
         asm volatile(
             "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
             : "=r"(ok)
-            : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
+            : "r"(smem_u32(bar)), "r"(parity), "r"(100000u)
             : "memory");
     return ok != 0;
 }
@@ -78,8 +78,10 @@ __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, vola
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait_t<CLUSTER>(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if ((i & 15u) == 15u && global_timer_ns() - t0 > 1000000000ull) break;
+        if ((i & 7u) == 7u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > 1000000000ull) break;
+        }
     }
     *abort_flag = 1;
     atomicExch(status, 5 /* DSLA_ERR_TIMEOUT */);
