@@ -390,7 +390,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "cfg5"])
     ap.add_argument("--dense", default=None, metavar="B,H,T", help="shape sweep: a dense bf16 d=128 batch instead of --workload")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "simt", "tensor", "pair"])
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-layers", type=int, default=0, help="layers in the decode section (0 = the workload's 32); "
                     "smaller stacks exist for profiler captures")

@@ -18,7 +18,9 @@
  *     stream) and the call returns without waiting for it;
  *   - argument errors are detected on the host before anything is launched and reported through
  *     the return value; nothing is thrown, nothing aborts, there is no CPU fallback;
- *   - supported head sizes: d_k == d_v in {64, 128}; everything else is DSLA_ERR_UNSUPPORTED.
+ *   - supported head sizes: d_k == d_v in {64, 128}; everything else is DSLA_ERR_UNSUPPORTED;
+ *   - a state store belongs to the device that was current in dsla_state_alloc; prefill and decode calls for it must be
+ *     made with that device current (DSLA_ERR_INVALID_ARG otherwise).
  */
 #ifndef DSLA_H_
 #define DSLA_H_
@@ -42,8 +44,14 @@ typedef enum {
 
 typedef enum { DSLA_F32 = 0, DSLA_BF16 = 1 } dsla_dtype;
 
-/* Which prefill kernel runs.  AUTO picks TENSOR for bf16 with d = 128 and SIMT otherwise. */
-typedef enum { DSLA_IMPL_AUTO = 0, DSLA_IMPL_SIMT = 1, DSLA_IMPL_TENSOR = 2 } dsla_impl;
+/* Which prefill kernel runs.
+ *   SIMT        : CUDA cores, fp32 arithmetic; any supported dtype and head size, chunk 16 / 32 / 64.
+ *   TENSOR      : tcgen05 tensor cores, bf16 with d = 128, chunk 64; one CTA holds both states of a (sequence, head) pair.
+ *   TENSOR_PAIR : same mathematics and limits, one state per CTA in a cluster of two CTAs that exchange partial
+ *                 outputs through distributed shared memory.
+ *   AUTO        : TENSOR for bf16 with d = 128 (the faster of the two tensor variants on the measured shapes), else SIMT
+ *                 -- in particular bf16 with d = 64 and everything fp32 run on CUDA cores, an order of magnitude slower. */
+typedef enum { DSLA_IMPL_AUTO = 0, DSLA_IMPL_SIMT = 1, DSLA_IMPL_TENSOR = 2, DSLA_IMPL_TENSOR_PAIR = 3 } dsla_impl;
 
 /* ------------------------------------------------------------------------------------------
  * Dual-state store.  One "slot" holds the two states of every head of one sequence of one layer:
@@ -193,7 +201,9 @@ dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cu
  * 2048 tokens or more (cu_seqlens == NULL, N == 1) is cut into slices of about 1024 tokens: while slice i is computed,
  * continuing from the states slice i-1 left in the slot, the inputs of slice i+1 and the outputs of slice i-1 are copied
  * on two internal streams (created once per device) that are forked from and joined back into `cuda_stream` with
- * events; the result equals the unsliced one up to floating-point summation order.
+ * events; the result equals the unsliced one up to floating-point summation order.  Those streams and events are one set
+ * per device: host threads that call dsla_prefill_host at the same time are enqueued one after the other (a mutex), and two
+ * calls on different caller streams must not be in flight on the GPU together (the second would wait on events the first recorded).
  * ------------------------------------------------------------------------------------------ */
 size_t dsla_prefill_staging_bytes(const dsla_prefill_args* a);
 dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* staging,

@@ -24,9 +24,9 @@ DSLA_OK, DSLA_ERR_INVALID_ARG, DSLA_ERR_UNSUPPORTED, DSLA_ERR_CUDA, DSLA_ERR_OOM
 DSLA_ERR_SCRATCH_LIMIT = 6
 DSLA_STATIC_SCRATCH_BYTES = 18 << 20
 DSLA_F32, DSLA_BF16 = 0, 1
-DSLA_IMPL_AUTO, DSLA_IMPL_SIMT, DSLA_IMPL_TENSOR = 0, 1, 2
+DSLA_IMPL_AUTO, DSLA_IMPL_SIMT, DSLA_IMPL_TENSOR, DSLA_IMPL_TENSOR_PAIR = 0, 1, 2, 3
 _DTYPES = {torch.float32: DSLA_F32, torch.bfloat16: DSLA_BF16}
-_IMPLS = {"auto": DSLA_IMPL_AUTO, "simt": DSLA_IMPL_SIMT, "tensor": DSLA_IMPL_TENSOR}
+_IMPLS = {"auto": DSLA_IMPL_AUTO, "simt": DSLA_IMPL_SIMT, "tensor": DSLA_IMPL_TENSOR, "pair": DSLA_IMPL_TENSOR_PAIR}
 
 
 class dsla_prefill_args(Structure):

@@ -23,6 +23,11 @@ __global__ void zero_slots_kernel(float* data, const int32_t* slots, int num_slo
 
 using namespace dsla;
 
+// A store belongs to the device that was current when it was created; kernels for it must be launched there.
+static bool on_store_device(const dsla_state* st) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == st->device;
+}
 static bool supported_d(int dk, int dv) { return dk == dv && (dk == 64 || dk == 128); }
 static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 static size_t esize(dsla_dtype dt) { return dt == DSLA_F32 ? 4 : 2; }
@@ -126,7 +131,7 @@ dsla_status dsla_selftest_bounded_wait(dsla_state* st, unsigned max_polls, void*
 
 // ---- prefill ------------------------------------------------------------------------------
 static dsla_impl resolve_impl(const dsla_prefill_args* a) {
-    if (a->impl == DSLA_IMPL_SIMT || a->impl == DSLA_IMPL_TENSOR) return a->impl;
+    if (a->impl == DSLA_IMPL_SIMT || a->impl == DSLA_IMPL_TENSOR || a->impl == DSLA_IMPL_TENSOR_PAIR) return a->impl;
     return (a->dtype == DSLA_BF16 && a->d_k == 128 && prefill_tc_available()) ? DSLA_IMPL_TENSOR : DSLA_IMPL_SIMT;
 }
 
@@ -141,7 +146,8 @@ static dsla_status check_prefill_sizes(const dsla_prefill_args* a) {
     } else if (a->max_seqlen > a->T_total) {
         return DSLA_ERR_INVALID_ARG;
     }
-    if (a->impl != DSLA_IMPL_AUTO && a->impl != DSLA_IMPL_SIMT && a->impl != DSLA_IMPL_TENSOR) return DSLA_ERR_INVALID_ARG;
+    if (a->impl != DSLA_IMPL_AUTO && a->impl != DSLA_IMPL_SIMT && a->impl != DSLA_IMPL_TENSOR && a->impl != DSLA_IMPL_TENSOR_PAIR)
+        return DSLA_ERR_INVALID_ARG;
     const dsla_impl impl = resolve_impl(a);
     const int chunk = a->chunk == 0 ? 64 : a->chunk;
     if (impl == DSLA_IMPL_SIMT) {
@@ -154,7 +160,8 @@ static dsla_status check_prefill_sizes(const dsla_prefill_args* a) {
 
 size_t dsla_prefill_workspace_bytes(const dsla_prefill_args* a) {
     if (check_prefill_sizes(a) != DSLA_OK) return 0;
-    return resolve_impl(a) == DSLA_IMPL_TENSOR ? prefill_tc_workspace_bytes(a) : 0;
+    const dsla_impl impl = resolve_impl(a);
+    return impl == DSLA_IMPL_SIMT ? 0 : prefill_tc_workspace_bytes(a, impl == DSLA_IMPL_TENSOR_PAIR);
 }
 
 static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cudaStream_t s) {
@@ -163,6 +170,7 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     if (!st) return DSLA_ERR_INVALID_ARG;
     if (st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
     if (!a->slots && a->N > st->num_slots) return DSLA_ERR_INVALID_ARG;
+    if (!on_store_device(st)) return DSLA_ERR_INVALID_ARG;
     if (a->N == 0) return DSLA_OK;
     if (!a->gamma) return DSLA_ERR_INVALID_ARG;
     if (a->T_total > 0) {
@@ -183,7 +191,8 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     const int chunk = a->chunk == 0 ? 64 : a->chunk;
     p.max_chunks = (a->max_seqlen + chunk - 1) / chunk;
     p.scale = a->scale; p.use_initial_state = a->use_initial_state ? 1 : 0;
-    if (resolve_impl(a) == DSLA_IMPL_TENSOR) return launch_prefill_tc(p, a, s);
+    const dsla_impl impl = resolve_impl(a);
+    if (impl != DSLA_IMPL_SIMT) return launch_prefill_tc(p, a, impl == DSLA_IMPL_TENSOR_PAIR, s);
     return launch_prefill_simt(p, a->d_k, chunk, a->dtype, s);
 }
 
@@ -206,6 +215,7 @@ static dsla_status check_decode(const dsla_decode_args* a, dsla_state* st) {
     if (st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
     if (!a->slots && a->B > st->num_slots) return DSLA_ERR_INVALID_ARG;
     if (!(a->scale == a->scale)) return DSLA_ERR_INVALID_ARG;
+    if (!on_store_device(st)) return DSLA_ERR_INVALID_ARG;
     return DSLA_OK;
 }
 
@@ -272,6 +282,9 @@ HostPipe* host_pipe() {
 dsla_status prefill_host_sliced(const dsla_prefill_args* a, const dsla_prefill_args& d, dsla_state* st, cudaStream_t s) {
     HostPipe* hp = host_pipe();
     if (!hp) return DSLA_ERR_CUDA;
+    // The side streams and events are one set per device: calls from several host threads enqueue one after the other.
+    static std::mutex enqueue_mutex;
+    std::lock_guard<std::mutex> enqueue_lock(enqueue_mutex);
     const int T = a->T_total;
     int nsl = T / 1024;
     if (nsl > HOST_MAX_SLICES) nsl = HOST_MAX_SLICES;
@@ -298,7 +311,12 @@ dsla_status prefill_host_sliced(const dsla_prefill_args* a, const dsla_prefill_a
         sl.T = len; sl.T_total = len; sl.max_seqlen = len;
         sl.use_initial_state = i > 0 ? 1 : a->use_initial_state;
         const dsla_status rc = prefill_device(&sl, st, s);
-        if (rc != DSLA_OK) return rc;
+        if (rc != DSLA_OK) {
+            // join the forked side streams back into the caller's stream before reporting the failure
+            if (cudaEventRecord(hp->end, hp->h2d) == cudaSuccess) (void)cudaStreamWaitEvent(s, hp->end, 0);
+            if (cudaEventRecord(hp->end, hp->d2h) == cudaSuccess) (void)cudaStreamWaitEvent(s, hp->end, 0);
+            return rc;
+        }
         ok = cudaEventRecord(hp->done[i], s) == cudaSuccess && cudaStreamWaitEvent(hp->d2h, hp->done[i], 0) == cudaSuccess &&
              cudaMemcpyAsync(dev(a->o, off), dev(d.o, off), nb, cudaMemcpyDeviceToHost, hp->d2h) == cudaSuccess;
     }

@@ -51,10 +51,10 @@ dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStrea
 dsla_status launch_prefill_simt(const PrefillParams& p, int d, int chunk, dsla_dtype dt, cudaStream_t s);
 // dsla_prefill_summary.cu: one warp waits, with the given poll limit, on a barrier nobody arrives at
 void launch_bounded_wait_selftest(int* status, unsigned max_polls, cudaStream_t s);
-// dsla_prefill_tc.cu
+// dsla_prefill_tc.cu (pair = the cluster variant of dsla_prefill_tc_pair.cu)
 bool prefill_tc_available();
-size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a);
-dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a, cudaStream_t s);
+size_t prefill_tc_workspace_bytes(const dsla_prefill_args* a, bool pair);
+dsla_status launch_prefill_tc(const PrefillParams& p, const dsla_prefill_args* a, bool pair, cudaStream_t s);
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }

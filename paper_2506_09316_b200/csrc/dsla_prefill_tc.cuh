@@ -127,8 +127,9 @@ bool make_tile_map(CUtensorMap* m, const void* base, int T_total, int H);
 void launch_seq_order(const int32_t* cu, int N, int* order, cudaStream_t s);
 void launch_state_snapshot(const PrefillParams& p, float* snap, cudaStream_t s);
 dsla_status launch_summary(const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& tp, cudaStream_t s);
-// dsla_prefill_tc_v1.cu: the earlier main kernel (both states in one CTA), kept for comparison runs
-dsla_status launch_main_v1(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& tp, bool dependent,
-                           cudaStream_t s);
+// dsla_prefill_tc_pair.cu: the cluster variant's main grid, and how many of its clusters fit on the device at once
+dsla_status launch_main_pair(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const TcParams& tp, bool dependent,
+                             cudaStream_t s);
+int pair_resident_clusters();
 
 }  // namespace dsla

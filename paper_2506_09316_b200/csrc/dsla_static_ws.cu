@@ -1,6 +1,8 @@
 // dsla_prefill_static_ws: prefill for callers that cannot supply (or allocate) a scratch buffer.
 // The scratch lives in a fixed device array that is part of the library image, so the call path
 // contains no allocation at all.
+#include <atomic>
+
 #include "dsla_internal.cuh"
 
 namespace {
@@ -11,23 +13,23 @@ namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[DSLA_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices];   // device address of the array on each device, filled on first use
-bool g_scratch_known[kMaxDevices];
+// device address of the array on each device, filled on first use; two host threads that race on the first call both
+// look the address up and store the same value
+std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 // Device address of the scratch array on the current device (looked up once per device).
 dsla_status static_scratch(void** out) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DSLA_ERR_CUDA;
-    if (!g_scratch_known[dev]) {
-        void* ptr = nullptr;
+    void* ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (ptr == nullptr) {
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
             (void)cudaGetLastError();
             return DSLA_ERR_CUDA;
         }
-        g_scratch_addr[dev] = ptr;
-        g_scratch_known[dev] = true;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = ptr;
     return DSLA_OK;
 }
 

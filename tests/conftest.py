@@ -33,3 +33,9 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(params=["tensor", "pair"])
+def tc_impl(request):
+    """Both tensor-core prefill variants: both states in one CTA / one state per CTA of a two-CTA cluster."""
+    return request.param

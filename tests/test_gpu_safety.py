@@ -54,3 +54,22 @@ def test_sequence_longer_than_max_seqlen_is_reported(H):
     assert dsla.dsla_state_last_error(st) == dsla.DSLA_OK
     o_ref, _ = oracle_prefill(inp)
     assert rel_err(o.double().cpu().numpy(), o_ref) <= TOL[BF]
+
+
+def test_split_prefill_with_initial_state_next_to_a_busy_stream(tc_impl):
+    """A sequence split into segments that resumes from a stored state: the CTA of the last segment overwrites the slot
+    that CTAs of earlier segments read as their initial state.  They read a snapshot taken beforehand, so the result must
+    not depend on how the CTAs get scheduled -- here a second stream keeps part of the GPU busy with ordinary matmuls."""
+    import paper_2506_09316_b200 as dsla
+    inp = gen.make_dense(9903, 1, 64 * 48, 2, 128, BF)
+    st0 = gen.make_states(9904, 1, 2, 128, 128, std=0.4).numpy()
+    o_ref, S_ref = oracle_prefill(inp, state0=st0)
+    side = torch.cuda.Stream()
+    a = torch.randn(4096, 4096, device="cuda", dtype=torch.bfloat16)
+    for attempt in range(3):
+        with torch.cuda.stream(side):
+            for _ in range(6):
+                a @ a                                  # bounded, ordinary work that occupies SMs for a while
+        o, S = gpu_prefill(inp, state0=st0, impl=tc_impl)
+        side.synchronize()
+        assert rel_err(o, o_ref) <= TOL[BF] and rel_err(S, S_ref) <= TOL[BF], f"attempt {attempt}"

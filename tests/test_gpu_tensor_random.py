@@ -13,7 +13,7 @@ BF = torch.bfloat16
 
 
 @pytest.mark.parametrize("case", range(12))
-def test_tensor_prefill_random_case(case):
+def test_tensor_prefill_random_case(case, tc_impl):
     rng = np.random.default_rng(9100 + case)
     H = int(rng.choice([1, 2, 3, 5, 8, 40]))
     N = int(rng.integers(1, 5 if H == 40 else 7))
@@ -37,7 +37,7 @@ def test_tensor_prefill_random_case(case):
     use_init = bool(rng.integers(0, 2))
     slots = [int(x) for x in rng.permutation(N + 2)[:N]]
     st0 = gen.make_states(9300 + case, N + 2, H, 128, 128, std=0.3).numpy() if use_init else None
-    kw = dict(state0=st0, slots=slots, num_slots=N + 2, impl="tensor", scale=0.7)
+    kw = dict(state0=st0, slots=slots, num_slots=N + 2, impl=tc_impl, scale=0.7)
     o, S = gpu_prefill(inp, **kw)
     o2, S2 = gpu_prefill(inp, **kw)
     assert np.array_equal(o, o2) and all(np.array_equal(S[s], S2[s]) for s in slots), "not reproducible"
