@@ -22,6 +22,13 @@
  * Pins (tests/test_oracle_pins.py): quadratic masked form built from explicit gate products,
  * unrolled score form, single-state (GLA) reduction, g = 1 cumulative-sum form, g = 0 form,
  * geometric-series closed form, composition, chunked restatement, linearity, permutation.
+ *
+ * dsla_oracle_run_n is the same loop for n states with one blend weight per state (the generalisation
+ * to more than two states of Sec. 4.2, run with 1, 2, 4 and 8 states in the number-of-states ablation
+ * of Sec. 5.5):   S^i_t = G^i_t (.) S^i_{t-1} + k_t^T v_t,   o_t = q_t sum_i w_i S^i_t.
+ * Pins (tests/test_oracle_nstate.py): unrolled score form with explicit gate products for 1, 3, 4 states;
+ * two states with w = (gamma, 1 - gamma) reproduce dsla_oracle_run bit for bit; one state is the plain
+ * gated-linear-attention loop of Sec. 3.
  */
 #include <pthread.h>
 #include <stdint.h>
@@ -110,6 +117,85 @@ int dsla_oracle_run(const double *q, const double *k, const double *v,
     } else {
         pthread_t *th = (pthread_t *)malloc(sizeof(pthread_t) * (size_t)nthreads);
         for (int i = 0; i < nthreads; ++i) pthread_create(&th[i], NULL, worker, &J);
+        for (int i = 0; i < nthreads; ++i) pthread_join(th[i], NULL);
+        free(th);
+    }
+    pthread_mutex_destroy(&J.mu);
+    return 0;
+}
+
+
+/* ---- n states ------------------------------------------------------------------------------- */
+typedef struct {
+    const double *q, *k, *v;
+    const double *const *g;       /* n pointers: [T_total, H] or [T_total, H, dk] when per_channel */
+    const double *w;              /* [H, n] blend weight of every state */
+    const int32_t *cu, *slots;
+    int N, H, dk, dv, n, per_channel;
+    double scale;
+    double *S;                    /* [num_slots, n, H, dk, dv] in/out */
+    double *o;
+    int next_unit;
+    pthread_mutex_t mu;
+} jobn_t;
+
+static void run_unit_n(const jobn_t *J, int s, int h)
+{
+    const int H = J->H, dk = J->dk, dv = J->dv, n = J->n;
+    const int slot = J->slots ? J->slots[s] : s;
+    if (slot < 0) return;
+    for (int t = J->cu[s]; t < J->cu[s + 1]; ++t) {
+        const double *qt = J->q + ((size_t)t * H + h) * dk;
+        const double *kt = J->k + ((size_t)t * H + h) * dk;
+        const double *vt = J->v + ((size_t)t * H + h) * dv;
+        double *ot = J->o + ((size_t)t * H + h) * dv;
+        for (int b = 0; b < dv; ++b) ot[b] = 0.0;
+        for (int i = 0; i < n; ++i) {
+            double *Si = J->S + (((size_t)slot * n + i) * H + h) * (size_t)dk * dv;
+            const double wi = J->w[(size_t)h * n + i];
+            for (int a = 0; a < dk; ++a) {
+                const double g = J->per_channel ? J->g[i][((size_t)t * H + h) * dk + a] : J->g[i][(size_t)t * H + h];
+                double *row = Si + (size_t)a * dv;
+                for (int b = 0; b < dv; ++b) {
+                    row[b] = g * row[b] + kt[a] * vt[b];          /* S^i_t = G^i_t (.) S^i_{t-1} + k_t^T v_t */
+                    ot[b] += qt[a] * wi * row[b];                 /* o_t = q_t sum_i w_i S^i_t */
+                }
+            }
+        }
+        for (int b = 0; b < dv; ++b) ot[b] *= J->scale;
+    }
+}
+
+static void *worker_n(void *p)
+{
+    jobn_t *J = (jobn_t *)p;
+    for (;;) {
+        pthread_mutex_lock(&J->mu);
+        int u = J->next_unit++;
+        pthread_mutex_unlock(&J->mu);
+        if (u >= J->N * J->H) break;
+        run_unit_n(J, u / J->H, u % J->H);
+    }
+    return NULL;
+}
+
+int dsla_oracle_run_n(const double *q, const double *k, const double *v, const double *const *gates, int n_states,
+                      int per_channel, const double *weights, const int32_t *cu_seqlens, const int32_t *slots,
+                      int N, int H, int dk, int dv, double scale, double *S, double *o, int nthreads)
+{
+    if (N < 0 || H <= 0 || dk <= 0 || dv <= 0 || n_states <= 0 || !cu_seqlens) return -1;
+    jobn_t J;
+    memset(&J, 0, sizeof J);
+    J.q = q; J.k = k; J.v = v; J.g = gates; J.w = weights; J.cu = cu_seqlens; J.slots = slots;
+    J.N = N; J.H = H; J.dk = dk; J.dv = dv; J.n = n_states; J.per_channel = per_channel; J.scale = scale; J.S = S; J.o = o;
+    pthread_mutex_init(&J.mu, NULL);
+    if (nthreads < 1) nthreads = 1;
+    if (nthreads > N * H) nthreads = N * H > 0 ? N * H : 1;
+    if (nthreads == 1) {
+        worker_n(&J);
+    } else {
+        pthread_t *th = (pthread_t *)malloc(sizeof(pthread_t) * (size_t)nthreads);
+        for (int i = 0; i < nthreads; ++i) pthread_create(&th[i], NULL, worker_n, &J);
         for (int i = 0; i < nthreads; ++i) pthread_join(th[i], NULL);
         free(th);
     }
