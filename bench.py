@@ -137,16 +137,40 @@ def workload_spec(name, dense=None):
 
 
 # --------------------------------------------------------------------------------------------
-def bench_ours(args):
-    import paper_2506_09316_b200 as dsla
-    rank, world, local = dist_env()
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    peaks = load_peaks()
-    spec = workload_spec(args.workload, args.dense)
+KERNEL_SOURCES = {   # the files whose change makes a stored DRAM-traffic figure stale
+    "tensor": ["dsla_prefill_tc.cu", "dsla_prefill_summary.cu", "dsla_prefill_tc.cuh", "tc_utils.cuh"],
+    "pair": ["dsla_prefill_tc_pair.cu", "dsla_prefill_summary.cu", "dsla_prefill_tc.cuh", "tc_utils.cuh"],
+    "decode": ["dsla_decode.cu"],
+}
+
+
+def source_digest(kind):
+    import hashlib
+    h = hashlib.sha1()
+    for f in KERNEL_SOURCES[kind]:
+        h.update(open(os.path.join(ROOT, "paper_2506_09316_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:12]
+
+
+def stored_traffic(kernel, workload):
+    """DRAM bytes per launch from the table of ncu captures kept with the profile summaries; None when there is no
+    row for this kernel and workload or when the kernel's sources have changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.md")
+    if not os.path.exists(path):
+        return None
+    for line in open(path):
+        cells = [c.strip() for c in line.strip().strip("|").split("|")]
+        if len(cells) >= 4 and cells[0] == kernel and cells[1] == workload:
+            try:
+                return float(cells[2]) if cells[3] == source_digest(kernel) else None
+            except ValueError:
+                return None
+    return None
+
+
+def time_prefill(dsla, spec, kernel, steps, warmup, dev, rank, peaks, with_decode_leg=False, min_seconds=0.0):
+    """Times `steps` prefills of one workload (CUDA events per step on the launching stream, rotating input sets larger
+    than L2).  With min_seconds the timed region is repeated until it has lasted that long (sustained figure)."""
     H, d, lens = spec["H"], spec["d"], spec["lens"]
     N, T_total, max_len = len(lens), int(sum(lens)), int(max(lens))
     dense = len(set(lens)) == 1
@@ -156,10 +180,9 @@ def bench_ours(args):
             for i in range(n_sets)]
     outs = [torch.empty_like(s.v) for s in sets]
     st = dsla.dsla_state_alloc(N, H, d, d, device=dev)
-    ws_bytes = dsla.binding.dsla_prefill_workspace_bytes(T_total, N, max_len, H, d, torch.bfloat16, 64, args.kernel,
+    ws_bytes = dsla.binding.dsla_prefill_workspace_bytes(T_total, N, max_len, H, d, torch.bfloat16, 64, kernel,
                                                         dense_T=max_len if dense else None)
     ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device=dev) if ws_bytes else None
-    # decode inputs for the step's decode leg: one token per sequence
     dec = gen.make_packed_device(spec["seed"] + 5, [1] * N, H, d, torch.bfloat16, device=dev)
     dec_o = torch.empty_like(dec.v)
     stream = torch.cuda.current_stream()
@@ -170,17 +193,81 @@ def bench_ours(args):
             ev[0].record(stream)
         dsla.dsla_prefill(s.q, s.k, s.v, s.g_hist, s.g_rec, s.gamma, st, o=outs[i % n_sets],
                           cu_seqlens=None if dense else s.cu_seqlens, max_seqlen=max_len, chunk=64,
-                          impl=args.kernel, workspace=ws)
+                          impl=kernel, workspace=ws)
         if ev:
             ev[1].record(stream)
-        dsla.dsla_decode_step(dec.q, dec.k, dec.v, dec.g_hist, dec.g_rec, s.gamma, st, o=dec_o)
+        if with_decode_leg:
+            dsla.dsla_decode_step(dec.q, dec.k, dec.v, dec.g_hist, dec.g_rec, s.gamma, st, o=dec_o)
         if ev:
             ev[2].record(stream)
 
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(i)
     torch.cuda.synchronize()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    res = dict(sets=sets, dec=dec, st=st, ws=ws, lens=lens, dense=dense, max_len=max_len, n_sets=n_sets,
+               bytes_per_set=bytes_per_set, T_total=T_total, N=N, step=step)
+    if min_seconds > 0:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 0
+        e0.record(stream)
+        t_host = time.perf_counter()
+        while True:
+            for i in range(steps):
+                step(n + i)
+            n += steps
+            if n % (8 * steps) == 0:
+                stream.synchronize()          # bound the launch queue; the GPU stays busy between checks for < 1 %
+            if time.perf_counter() - t_host >= min_seconds:
+                break
+        e1.record(stream)
+        torch.cuda.synchronize()
+        res.update(n=n, total_ms=e0.elapsed_time(e1))
+        return res
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    res["evs"] = evs
+    return res
+
+
+def prefill_numbers(T_total, H, d, ms, peaks, world=1):
+    flops = T_total * H * FLOP_PER_TOKEN_HEAD(d, 64)
+    nbytes = T_total * H * PREFILL_BYTES_PER_TOKEN_HEAD(d, 2)
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"ms": ms, "tokens_per_s": world * T_total / (ms * 1e-3), "tflops": tf, "frac": tf / peaks["bf16_tflops"],
+            "hbm_gbs": nbytes / (ms * 1e-3) / 1e9, "hbm_frac": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+
+def extra_prefill_section(dsla, name, kernel, steps, dev, rank, peaks, dense=None):
+    """A further prefill workload reported beside the headline one: median and best of the per-step event times."""
+    spec = workload_spec(name, dense)
+    r = time_prefill(dsla, spec, kernel, steps, 3, dev, rank, peaks)
+    stream = torch.cuda.current_stream()
+    for i in range(steps):
+        r["step"](i, r["evs"][i])
+    torch.cuda.synchronize()
+    ms = [e[0].elapsed_time(e[1]) for e in r["evs"]]
+    out = {"workload": f"{dense or name}: N={r['N']} H={spec['H']} d={spec['d']} T_total={r['T_total']}", "kernel": kernel, "steps": steps,
+           "median": prefill_numbers(r["T_total"], spec["H"], spec["d"], float(np.median(ms)), peaks),
+           "best": prefill_numbers(r["T_total"], spec["H"], spec["d"], float(np.min(ms)), peaks)}
+    del r
+    torch.cuda.empty_cache()
+    return out
+
+
+def bench_ours(args):
+    import paper_2506_09316_b200 as dsla
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    spec = workload_spec(args.workload, args.dense)
+    H, d = spec["H"], spec["d"]
+    r = time_prefill(dsla, spec, args.kernel, args.steps, args.warmup, dev, rank, peaks, with_decode_leg=True)
+    sets, dec, st, ws, lens, dense, max_len = r["sets"], r["dec"], r["st"], r["ws"], r["lens"], r["dense"], r["max_len"]
+    N, T_total, n_sets, bytes_per_set, evs, step = r["N"], r["T_total"], r["n_sets"], r["bytes_per_set"], r["evs"], r["step"]
+    stream = torch.cuda.current_stream()
     sampler = ClockSampler(visible_nvml_index(local))
     barrier(world)
     torch.cuda.synchronize()
@@ -197,31 +284,61 @@ def bench_ours(args):
     barrier(world)
     launches = dsla.dsla_launch_count() - launches0
     total_ms = max_over_ranks(t_start.elapsed_time(t_stop), world, dev)
-    prefill_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    per_step = [e[0].elapsed_time(e[1]) for e in evs]
+    prefill_ms = float(np.mean(per_step))
     decode_leg_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     ms_per_step = total_ms / args.steps
     tokens_per_step = T_total + N
     value = world * tokens_per_step / (ms_per_step * 1e-3)
 
-    flops = T_total * H * FLOP_PER_TOKEN_HEAD(d, 64)
-    achieved_tf = flops / (prefill_ms * 1e-3) / 1e12
-    # DRAM bytes per prefill (main + summary kernel) from one ncu capture of this workload; its summary is kept with the other profiles
-    traffic = 181.0e6 if (args.workload == "cfg2" and not args.dense and args.kernel != "simt") else None
-    roofline = {"kernel": "prefill (summary + main launch)", "bound": "tensor", "achieved": achieved_tf, "peak": peaks["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": achieved_tf / peaks["bf16_tflops"], "traffic": traffic,
-                "algorithmic_bytes": bytes_per_set, "algorithmic_flops": flops,
+    kernel_name = "pair" if args.kernel == "pair" else "tensor"
+    pn = prefill_numbers(T_total, H, d, prefill_ms, peaks)
+    traffic = stored_traffic(kernel_name, args.dense or args.workload) if args.kernel != "simt" else None
+    roofline = {"kernel": f"prefill ({'summary + ' if N * H < 148 else ''}main launch, --kernel {args.kernel})", "bound": "tensor",
+                "achieved": pn["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": pn["frac"], "traffic": traffic,
+                "algorithmic_bytes": bytes_per_set, "algorithmic_flops": T_total * H * FLOP_PER_TOKEN_HEAD(d, 64),
                 "peak_source": f"{peaks['source']} burst bf16 (kernel timed alone between events)",
-                "hbm_gbs": bytes_per_set / (prefill_ms * 1e-3) / 1e9,
-                "hbm_frac": bytes_per_set / (prefill_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                "hbm_gbs": pn["hbm_gbs"], "hbm_frac": pn["hbm_frac"],
+                "median_ms": float(np.median(per_step)), "best_ms": float(np.min(per_step))}
+
+    # ---- the same prefill repeated for at least half a second in one timed region (clocks and power settle)
+    sustained = None
+    if not args.no_sustained:
+        sampler2 = ClockSampler(visible_nvml_index(local))
+        sampler2.start()
+        rs = time_prefill(dsla, spec, args.kernel, 16, 3, dev, rank, peaks, min_seconds=args.sustained_seconds)
+        ck = sampler2.stop()
+        ms = max_over_ranks(rs["total_ms"], world, dev) / rs["n"]
+        pn2 = prefill_numbers(T_total, H, d, ms, peaks, world)
+        sustained = {"seconds": rs["total_ms"] * 1e-3, "prefills": rs["n"], "ms": ms, "tokens_per_s": pn2["tokens_per_s"],
+                     "tflops": pn2["tflops"], "peak": peaks["bf16_tflops_sustained"], "frac": pn2["tflops"] / peaks["bf16_tflops_sustained"],
+                     "peak_source": f"{peaks['source']} sustained bf16", "clocks": ck}
+        del rs
 
     # ---- end to end through the host-buffer entry points (pinned host memory)
     e2e = None
     if not args.no_e2e:
         e2e = bench_e2e(dsla, sets[0], dec, st, ws, lens, dense, max_len, args, world, dev)
+    del r, sets, dec, st, ws, step, evs
+    torch.cuda.empty_cache()
+
+    # ---- the other prefill workloads and the other tensor-core variant (rank 0 reports; every rank runs them)
+    more = None
+    if not args.no_more:
+        more = {}
+        other = "pair" if args.kernel != "pair" else "tensor"
+        if not args.dense:
+            more[f"{args.workload}_{other}"] = extra_prefill_section(dsla, args.workload, other, 10, dev, rank, peaks)
+        for name in ("cfg3", "cfg5"):
+            if name != args.workload or args.dense:
+                more[name] = extra_prefill_section(dsla, name, args.kernel, 5, dev, rank, peaks)
+        more["dense_4x37x16384"] = extra_prefill_section(dsla, "cfg2", args.kernel, 5, dev, rank, peaks, dense="4,37,16384")
 
     decode = None
     if not args.no_decode:
         decode = bench_decode(dsla, args, peaks, world, dev, rank)
+        if not args.no_more:
+            decode["n_states"] = bench_decode_nstate(dsla, peaks, dev, rank)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -238,7 +355,8 @@ def bench_ours(args):
                        "parallelism": f"replicated x{world} (independent sequences, no collective)"},
             "prefill_only": {"value": world * T_total / (prefill_ms * 1e-3), "unit": "tokens/s (one layer)", "ms": prefill_ms},
             "decode_leg_ms": decode_leg_ms,
-            "roofline": roofline, "decode": decode, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "roofline": roofline, "prefill_sustained": sustained, "prefill_more": more, "decode": decode,
+            "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
         }
         print(json.dumps(line))
@@ -324,9 +442,55 @@ def bench_decode(dsla, args, peaks, world, dev, rank):
             "layer_tokens_per_s": world * B * steps * L / (ms * 1e-3), "ms_per_step": ms / steps,
             "gpu_launches": steps * L,
             "roofline": {"kernel": "decode", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": 1021.9e6 if B == 128 else None,  # profiles/decode_kernel_cfg4.md
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": stored_traffic("decode", "cfg4") if B == 128 else None,
                          "algorithmic_bytes": bytes_launch, "peak_source": f"{peaks['source']} copy bandwidth",
                          "us_per_launch": per_launch_s * 1e6}}
+
+
+def bench_decode_nstate(dsla, peaks, dev, rank):
+    """Decode step of the n-state form, n = 1, 2, 4, 8: B=128, H=32, d=128, a stack of layers whose states total
+    about 4 GB (>> L2), 32 steps; bytes per launch = n d^2 8 + inputs, against the measured copy bandwidth."""
+    c = gen.CONFIGS["cfg4"]
+    B, H, d = c["B"], c["H"], c["d"]
+    out = {}
+    for n in (1, 2, 4, 8):
+        per_layer = B * n * H * d * d * 4
+        L = max(2, int(4e9 // per_layer))
+        states = [dsla.dsla_state_alloc_n(B, n, H, d, d, device=dev) for _ in range(L)]
+        g = torch.Generator(device=dev)
+        g.manual_seed(c["seed"] + 31 * n + rank)
+        for s in states:
+            s.tensor.normal_(0.0, c["state_std"], generator=g)
+        inp = gen.make_packed_device(c["seed"] + 7 * n + rank, [1] * (L * B), H, d, torch.bfloat16, device=dev)
+        view = lambda t: t.view(L, B, *t.shape[1:])
+        q, k, v = map(view, (inp.q, inp.k, inp.v))
+        gates = torch.sigmoid(torch.randn((L, n, B, H), generator=g, device=dev) * 0.5 + 3.0)
+        w = torch.rand((H, n), generator=g, device=dev)
+        o = torch.empty_like(v)
+        stream = torch.cuda.current_stream()
+        steps = 32
+
+        def step():
+            for l in range(L):
+                dsla.dsla_nstate_decode_step(q[l], k[l], v[l], gates[l], w, states[l], o=o[l])
+
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        per_launch_s = e0.elapsed_time(e1) * 1e-3 / (steps * L)
+        nbytes = B * H * (2 * n * d * d * 4 + 4 * d * 2 + 4 * n)
+        gbs = nbytes / per_launch_s / 1e9
+        out[str(n)] = {"layers": L, "us_per_launch": per_launch_s * 1e6, "algorithmic_bytes": nbytes, "achieved": gbs,
+                       "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"]}
+        del states, inp, q, k, v, gates, o
+        torch.cuda.empty_cache()
+    return out
 
 
 # --------------------------------------------------------------------------------------------
@@ -395,6 +559,9 @@ def main():
     ap.add_argument("--decode-layers", type=int, default=0, help="layers in the decode section (0 = the workload's 32); "
                     "smaller stacks exist for profiler captures")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sustained-seconds", type=float, default=0.6)
+    ap.add_argument("--no-sustained", action="store_true")
+    ap.add_argument("--no-more", action="store_true", help="skip the further prefill workloads and the n-state decode section")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

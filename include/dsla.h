@@ -44,6 +44,11 @@ typedef enum {
 
 typedef enum { DSLA_F32 = 0, DSLA_BF16 = 1 } dsla_dtype;
 
+/* Shape of a gate tensor.  SCALAR: one activated gate per (token, head, state), G = g 11^T, shape [T, H].
+ * PER_KEY_CHANNEL: one gate per key channel, G = alpha^T 1 (the gated-linear-attention parameterisation of Sec. 2,
+ * which Sec. 4.1 carries over to G^1_t, G^2_t): shape [T, H, d_k]; row a of a state decays with alpha_a. */
+typedef enum { DSLA_GATE_SCALAR = 0, DSLA_GATE_PER_KEY_CHANNEL = 1 } dsla_gate_layout;
+
 /* Which prefill kernel runs.
  *   SIMT        : CUDA cores, fp32 arithmetic; any supported dtype and head size, chunk 16 / 32 / 64.
  *   TENSOR      : tcgen05 tensor cores, bf16 with d = 128, chunk 64; one CTA holds both states of a (sequence, head) pair.
@@ -130,6 +135,9 @@ typedef struct {
     dsla_impl impl;
     void* workspace;            /* scratch of dsla_prefill_workspace_bytes(); may be NULL if 0    */
     size_t workspace_bytes;
+    dsla_gate_layout gate_layout; /* SCALAR (0): g_hist, g_rec are [T_total, H].  PER_KEY_CHANNEL: [T_total, H, d_k];
+                                   served by a token-by-token CUDA-core kernel (impl AUTO or SIMT; the tensor-core
+                                   kernels take scalar gates only: DSLA_ERR_UNSUPPORTED)                        */
 } dsla_prefill_args;
 
 /* Scratch the chosen kernel needs for these sizes (0 for the SIMT kernel): the segment summaries of
@@ -188,9 +196,65 @@ typedef struct {
     int B, H, d_k, d_v;
     dsla_dtype dtype;
     float scale;
+    dsla_gate_layout gate_layout; /* SCALAR (0): g_hist, g_rec are [B, H]; PER_KEY_CHANNEL: [B, H, d_k]          */
+    const uint8_t* row_mask;    /* [B] bytes or NULL.  A batch may mix requests whose layer at this depth is a DSLA
+                                   layer with requests that still run softmax attention there (Sec. 4.5, App. D):
+                                   rows with 0 are not touched at all -- neither their slot nor their row of o, which
+                                   the attention kernel of the same step writes; NULL = every row is a DSLA row      */
 } dsla_decode_args;
 
 dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cuda_stream);
+
+/* ------------------------------------------------------------------------------------------
+ * n states.  Sec. 4.2 argues that two states suffice; the number-of-states ablation of Sec. 5.5 runs the layer with
+ * 1, 2, 4 and 8 states.  The general form keeps n recurrent states per (sequence, head), each with its own gate, and
+ * blends them with one weight per state:
+ *     S^i_t = g^i_t * S^i_{t-1} + k_t^T v_t   (i = 0 .. n-1),      o_t = scale * q_t sum_i w_i S^i_t .
+ * n = 2 with w = (gamma, 1 - gamma) is the dual-state layer above.  Supported n: 1, 2, 4, 8.
+ * The store is fp32 [num_slots][n_states][H][d_k][d_v]; dsla_state_alloc is dsla_state_alloc_n with n_states = 2, and
+ * the dual-state entry points accept only such stores (DSLA_ERR_INVALID_ARG otherwise).
+ * ------------------------------------------------------------------------------------------ */
+size_t dsla_state_bytes_n(int num_slots, int n_states, int H, int d_k, int d_v);
+dsla_status dsla_state_alloc_n(dsla_state** out, int num_slots, int n_states, int H, int d_k, int d_v,
+                               void* ext_buf, size_t ext_bytes);
+
+typedef struct {
+    const void* q;              /* [B, H, d_k] dtype                                                          */
+    const void* k;              /* [B, H, d_k]                                                                */
+    const void* v;              /* [B, H, d_v]                                                                */
+    void* o;                    /* [B, H, d_v] dtype (output)                                                 */
+    const float* gates;         /* [n_states, B, H] fp32 (or [n_states, B, H, d_k] per key channel)           */
+    const float* weights;       /* [H, n_states] fp32 blend weight of every state                             */
+    const int32_t* slots;       /* as in dsla_decode_args                                                     */
+    const uint8_t* row_mask;    /* as in dsla_decode_args                                                     */
+    int B, H, d_k, d_v, n_states;
+    dsla_dtype dtype;
+    float scale;
+    dsla_gate_layout gate_layout;
+} dsla_nstate_decode_args;
+
+/* One recurrence step of the n-state form, in place, one pass over the states (HBM traffic n_states/2 times that of
+ * the dual-state step). */
+dsla_status dsla_nstate_decode_step(const dsla_nstate_decode_args* a, dsla_state* st, void* cuda_stream);
+
+typedef struct {
+    const void *q, *k, *v;      /* [T_total, H, d] dtype, 16-byte aligned                                      */
+    void* o;                    /* [T_total, H, d_v] dtype (output)                                           */
+    const float* gates;         /* [n_states, T_total, H] fp32 (or [n_states, T_total, H, d_k])               */
+    const float* weights;       /* [H, n_states]                                                              */
+    const int32_t* cu_seqlens;  /* as in dsla_prefill_args                                                    */
+    const int32_t* slots;
+    int N, T, T_total, H, d_k, d_v, n_states;
+    dsla_dtype dtype;
+    float scale;
+    int use_initial_state;
+    dsla_gate_layout gate_layout;
+} dsla_nstate_prefill_args;
+
+/* Prefill of the n-state form on CUDA cores, token by token (fp32 arithmetic, no workspace).  With more than four
+ * states (more than two when the gates are per key channel and d = 128) the states are processed in groups, each group
+ * adding its share to o, so o is rounded to dtype once per group. */
+dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* st, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
  * Host-buffer variants (end-to-end path): q, k, v, o, g_hist, g_rec in `a` are HOST pointers

@@ -24,6 +24,7 @@ DSLA_OK, DSLA_ERR_INVALID_ARG, DSLA_ERR_UNSUPPORTED, DSLA_ERR_CUDA, DSLA_ERR_OOM
 DSLA_ERR_SCRATCH_LIMIT = 6
 DSLA_STATIC_SCRATCH_BYTES = 18 << 20
 DSLA_F32, DSLA_BF16 = 0, 1
+DSLA_GATE_SCALAR, DSLA_GATE_PER_KEY_CHANNEL = 0, 1
 DSLA_IMPL_AUTO, DSLA_IMPL_SIMT, DSLA_IMPL_TENSOR, DSLA_IMPL_TENSOR_PAIR = 0, 1, 2, 3
 _DTYPES = {torch.float32: DSLA_F32, torch.bfloat16: DSLA_BF16}
 _IMPLS = {"auto": DSLA_IMPL_AUTO, "simt": DSLA_IMPL_SIMT, "tensor": DSLA_IMPL_TENSOR, "pair": DSLA_IMPL_TENSOR_PAIR}
@@ -36,14 +37,29 @@ class dsla_prefill_args(Structure):
                 ("N", c_int), ("T", c_int), ("T_total", c_int), ("max_seqlen", c_int),
                 ("H", c_int), ("d_k", c_int), ("d_v", c_int), ("chunk", c_int),
                 ("dtype", c_int), ("scale", c_float), ("use_initial_state", c_int), ("impl", c_int),
-                ("workspace", c_void_p), ("workspace_bytes", c_size_t)]
+                ("workspace", c_void_p), ("workspace_bytes", c_size_t), ("gate_layout", c_int)]
 
 
 class dsla_decode_args(Structure):
     _fields_ = [("q", c_void_p), ("k", c_void_p), ("v", c_void_p), ("o", c_void_p),
                 ("g_hist", c_void_p), ("g_rec", c_void_p), ("gamma", c_void_p), ("slots", c_void_p),
                 ("B", c_int), ("H", c_int), ("d_k", c_int), ("d_v", c_int),
-                ("dtype", c_int), ("scale", c_float)]
+                ("dtype", c_int), ("scale", c_float), ("gate_layout", c_int), ("row_mask", c_void_p)]
+
+
+class dsla_nstate_decode_args(Structure):
+    _fields_ = [("q", c_void_p), ("k", c_void_p), ("v", c_void_p), ("o", c_void_p),
+                ("gates", c_void_p), ("weights", c_void_p), ("slots", c_void_p), ("row_mask", c_void_p),
+                ("B", c_int), ("H", c_int), ("d_k", c_int), ("d_v", c_int), ("n_states", c_int),
+                ("dtype", c_int), ("scale", c_float), ("gate_layout", c_int)]
+
+
+class dsla_nstate_prefill_args(Structure):
+    _fields_ = [("q", c_void_p), ("k", c_void_p), ("v", c_void_p), ("o", c_void_p),
+                ("gates", c_void_p), ("weights", c_void_p), ("cu_seqlens", c_void_p), ("slots", c_void_p),
+                ("N", c_int), ("T", c_int), ("T_total", c_int), ("H", c_int), ("d_k", c_int), ("d_v", c_int),
+                ("n_states", c_int), ("dtype", c_int), ("scale", c_float), ("use_initial_state", c_int),
+                ("gate_layout", c_int)]
 
 
 _lib.dsla_status_string.argtypes = [c_int]
@@ -54,6 +70,14 @@ _lib.dsla_state_bytes.argtypes = [c_int, c_int, c_int, c_int]
 _lib.dsla_state_bytes.restype = c_size_t
 _lib.dsla_state_alloc.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_void_p, c_size_t]
 _lib.dsla_state_alloc.restype = c_int
+_lib.dsla_state_bytes_n.argtypes = [c_int, c_int, c_int, c_int, c_int]
+_lib.dsla_state_bytes_n.restype = c_size_t
+_lib.dsla_state_alloc_n.argtypes = [POINTER(c_void_p), c_int, c_int, c_int, c_int, c_int, c_void_p, c_size_t]
+_lib.dsla_state_alloc_n.restype = c_int
+_lib.dsla_nstate_decode_step.argtypes = [POINTER(dsla_nstate_decode_args), c_void_p, c_void_p]
+_lib.dsla_nstate_decode_step.restype = c_int
+_lib.dsla_nstate_prefill.argtypes = [POINTER(dsla_nstate_prefill_args), c_void_p, c_void_p]
+_lib.dsla_nstate_prefill.restype = c_int
 _lib.dsla_state_free.argtypes = [c_void_p]
 _lib.dsla_state_free.restype = c_int
 _lib.dsla_state_data.argtypes = [c_void_p]
@@ -144,6 +168,23 @@ def dsla_state_alloc(num_slots: int, H: int, d_k: int, d_v: int, device="cuda", 
     return DslaState(h, buf, num_slots, H, d_k, d_v)
 
 
+def dsla_state_bytes_n(num_slots: int, n_states: int, H: int, d_k: int, d_v: int) -> int:
+    return int(_lib.dsla_state_bytes_n(num_slots, n_states, H, d_k, d_v))
+
+
+def dsla_state_alloc_n(num_slots: int, n_states: int, H: int, d_k: int, d_v: int, device="cuda") -> DslaState:
+    """Store of the n-state form; ``tensor`` is [num_slots, n_states, H, d_k, d_v] fp32."""
+    n = dsla_state_bytes_n(num_slots, n_states, H, d_k, d_v)
+    buf = torch.empty((num_slots, n_states, H, d_k, d_v), dtype=torch.float32, device=device) if n else None
+    h = c_void_p()
+    with torch.cuda.device(buf.device if buf is not None else device):
+        rc = _lib.dsla_state_alloc_n(byref(h), num_slots, n_states, H, d_k, d_v, _ptr(buf), n)
+    _check(rc, "dsla_state_alloc_n")
+    st = DslaState(h, buf, num_slots, H, d_k, d_v)
+    st.n_states = n_states
+    return st
+
+
 def dsla_state_free(st: DslaState):
     if st.handle is not None and st.handle.value:
         h, st.handle = st.handle, None
@@ -182,6 +223,7 @@ def _prefill_args(q, k, v, o, g_hist, g_rec, gamma, cu_seqlens, slots, N, T, max
     a.impl = _IMPLS[impl] if isinstance(impl, str) else int(impl)
     a.workspace = _ptr(workspace)
     a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a.gate_layout = DSLA_GATE_PER_KEY_CHANNEL if (g_hist is not None and g_hist.dim() == 3) else DSLA_GATE_SCALAR
     return a
 
 
@@ -249,7 +291,7 @@ def dsla_prefill_static_ws(q, k, v, g_hist, g_rec, gamma, st: DslaState, *, o=No
     return o
 
 
-def _decode_args(q, k, v, o, g_hist, g_rec, gamma, slots, scale):
+def _decode_args(q, k, v, o, g_hist, g_rec, gamma, slots, scale, row_mask=None):
     B, H, d_k = q.shape
     a = dsla_decode_args()
     a.q, a.k, a.v, a.o = _ptr(q), _ptr(k), _ptr(v), _ptr(o)
@@ -257,14 +299,18 @@ def _decode_args(q, k, v, o, g_hist, g_rec, gamma, slots, scale):
     a.B, a.H, a.d_k, a.d_v = int(B), int(H), int(d_k), int(v.shape[2])
     a.dtype = _DTYPES[q.dtype]
     a.scale = float(scale)
+    a.gate_layout = DSLA_GATE_PER_KEY_CHANNEL if g_hist.dim() == 3 else DSLA_GATE_SCALAR
+    a.row_mask = _ptr(row_mask)
     return a
 
 
-def dsla_decode_step(q, k, v, g_hist, g_rec, gamma, st: DslaState, *, o=None, slots=None, scale=1.0, stream=None):
-    """q, k, v: [B, H, d] device tensors; updates the rows' slots in place and returns o [B, H, d]."""
+def dsla_decode_step(q, k, v, g_hist, g_rec, gamma, st: DslaState, *, o=None, slots=None, scale=1.0, row_mask=None,
+                     stream=None):
+    """q, k, v: [B, H, d] device tensors; updates the rows' slots in place and returns o [B, H, d].  Gates [B, H], or
+    [B, H, d] per key channel.  ``row_mask`` (uint8 [B]): rows with 0 are not touched (state and o)."""
     if o is None:
         o = torch.empty_like(v)
-    a = _decode_args(q, k, v, o, g_hist, g_rec, gamma, slots, scale)
+    a = _decode_args(q, k, v, o, g_hist, g_rec, gamma, slots, scale, row_mask)
     _check(_lib.dsla_decode_step(byref(a), st.handle, _stream(stream)), "dsla_decode_step")
     return o
 
@@ -311,4 +357,45 @@ def dsla_decode_step_host(q, k, v, g_hist, g_rec, gamma, st: DslaState, o, stagi
     a = _decode_args(q, k, v, o, g_hist, g_rec, gamma, slots, scale)
     _check(_lib.dsla_decode_step_host(byref(a), st.handle, _ptr(staging), staging.numel() * staging.element_size(),
                                       _stream(stream)), "dsla_decode_step_host")
+    return o
+
+
+def dsla_nstate_decode_step(q, k, v, gates, weights, st: DslaState, *, o=None, slots=None, scale=1.0, row_mask=None,
+                            stream=None):
+    """n-state decode step: gates [n, B, H] (or [n, B, H, d] per key channel) fp32, weights [H, n] fp32."""
+    if o is None:
+        o = torch.empty_like(v)
+    B, H, d_k = q.shape
+    a = dsla_nstate_decode_args()
+    a.q, a.k, a.v, a.o = _ptr(q), _ptr(k), _ptr(v), _ptr(o)
+    a.gates, a.weights, a.slots, a.row_mask = _ptr(gates), _ptr(weights), _ptr(slots), _ptr(row_mask)
+    a.B, a.H, a.d_k, a.d_v, a.n_states = int(B), int(H), int(d_k), int(v.shape[2]), int(gates.shape[0])
+    a.dtype = _DTYPES[q.dtype]
+    a.scale = float(scale)
+    a.gate_layout = DSLA_GATE_PER_KEY_CHANNEL if gates.dim() == 4 else DSLA_GATE_SCALAR
+    _check(_lib.dsla_nstate_decode_step(byref(a), st.handle, _stream(stream)), "dsla_nstate_decode_step")
+    return o
+
+
+def dsla_nstate_prefill(q, k, v, gates, weights, st: DslaState, *, o=None, cu_seqlens=None, slots=None, max_seqlen=None,
+                        scale=1.0, use_initial_state=False, stream=None):
+    """n-state prefill (CUDA cores, token by token): gates [n, T_total, H] (or [n, T_total, H, d]), weights [H, n]."""
+    T_total, H, d_k = q.shape
+    if cu_seqlens is None:
+        T = int(max_seqlen) if max_seqlen is not None else T_total
+        N = T_total // T if T > 0 else 0
+    else:
+        N, T = cu_seqlens.numel() - 1, 0
+    if o is None:
+        o = torch.empty_like(v)
+    a = dsla_nstate_prefill_args()
+    a.q, a.k, a.v, a.o = _ptr(q), _ptr(k), _ptr(v), _ptr(o)
+    a.gates, a.weights, a.cu_seqlens, a.slots = _ptr(gates), _ptr(weights), _ptr(cu_seqlens), _ptr(slots)
+    a.N, a.T, a.T_total, a.H, a.d_k, a.d_v = int(N), int(T), int(T_total), int(H), int(d_k), int(v.shape[2])
+    a.n_states = int(gates.shape[0])
+    a.dtype = _DTYPES[q.dtype]
+    a.scale = float(scale)
+    a.use_initial_state = int(bool(use_initial_state))
+    a.gate_layout = DSLA_GATE_PER_KEY_CHANNEL if gates.dim() == 4 else DSLA_GATE_SCALAR
+    _check(_lib.dsla_nstate_prefill(byref(a), st.handle, _stream(stream)), "dsla_nstate_prefill")
     return o

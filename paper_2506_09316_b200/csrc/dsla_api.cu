@@ -49,21 +49,30 @@ const char* dsla_status_string(dsla_status s) {
 
 uint64_t dsla_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-size_t dsla_state_bytes(int num_slots, int H, int d_k, int d_v) {
-    if (num_slots <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return 0;
-    return (size_t)num_slots * 2 * (size_t)H * (size_t)d_k * (size_t)d_v * sizeof(float);
+static bool supported_n(int n) { return n == 1 || n == 2 || n == 4 || n == 8; }
+
+size_t dsla_state_bytes_n(int num_slots, int n_states, int H, int d_k, int d_v) {
+    if (num_slots <= 0 || n_states <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return 0;
+    return (size_t)num_slots * (size_t)n_states * (size_t)H * (size_t)d_k * (size_t)d_v * sizeof(float);
 }
 
+size_t dsla_state_bytes(int num_slots, int H, int d_k, int d_v) { return dsla_state_bytes_n(num_slots, 2, H, d_k, d_v); }
+
 dsla_status dsla_state_alloc(dsla_state** out, int num_slots, int H, int d_k, int d_v, void* ext_buf, size_t ext_bytes) {
+    return dsla_state_alloc_n(out, num_slots, 2, H, d_k, d_v, ext_buf, ext_bytes);
+}
+
+dsla_status dsla_state_alloc_n(dsla_state** out, int num_slots, int n_states, int H, int d_k, int d_v, void* ext_buf,
+                               size_t ext_bytes) {
     if (!out) return DSLA_ERR_INVALID_ARG;
     *out = nullptr;
-    if (num_slots <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return DSLA_ERR_INVALID_ARG;
-    if (!supported_d(d_k, d_v)) return DSLA_ERR_UNSUPPORTED;
-    const size_t bytes = dsla_state_bytes(num_slots, H, d_k, d_v);
+    if (num_slots <= 0 || n_states <= 0 || H <= 0 || d_k <= 0 || d_v <= 0) return DSLA_ERR_INVALID_ARG;
+    if (!supported_d(d_k, d_v) || !supported_n(n_states)) return DSLA_ERR_UNSUPPORTED;
+    const size_t bytes = dsla_state_bytes_n(num_slots, n_states, H, d_k, d_v);
     if (ext_buf && (ext_bytes < bytes || !aligned(ext_buf, 256))) return DSLA_ERR_INVALID_ARG;
     dsla_state* st = new (std::nothrow) dsla_state();
     if (!st) return DSLA_ERR_OOM;
-    st->num_slots = num_slots; st->H = H; st->d_k = d_k; st->d_v = d_v;
+    st->num_slots = num_slots; st->n_states = n_states; st->H = H; st->d_k = d_k; st->d_v = d_v;
     st->owns_data = ext_buf ? 0 : 1;
     st->data = static_cast<float*>(ext_buf);
     st->status = nullptr;
@@ -102,7 +111,7 @@ void* dsla_state_data(dsla_state* st) { return st ? st->data : nullptr; }
 dsla_status dsla_state_zero(dsla_state* st, const int32_t* slots_dev, int n, void* cuda_stream) {
     if (!st) return DSLA_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    const size_t slot_elems = (size_t)2 * st->H * st->d_k * st->d_v;
+    const size_t slot_elems = (size_t)st->n_states * st->H * st->d_k * st->d_v;
     if (!slots_dev) {
         return cudaMemsetAsync(st->data, 0, slot_elems * sizeof(float) * st->num_slots, s) == cudaSuccess ? DSLA_OK : DSLA_ERR_CUDA;
     }
@@ -131,6 +140,7 @@ dsla_status dsla_selftest_bounded_wait(dsla_state* st, unsigned max_polls, void*
 
 // ---- prefill ------------------------------------------------------------------------------
 static dsla_impl resolve_impl(const dsla_prefill_args* a) {
+    if (a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL) return DSLA_IMPL_SIMT;
     if (a->impl == DSLA_IMPL_SIMT || a->impl == DSLA_IMPL_TENSOR || a->impl == DSLA_IMPL_TENSOR_PAIR) return a->impl;
     return (a->dtype == DSLA_BF16 && a->d_k == 128 && prefill_tc_available()) ? DSLA_IMPL_TENSOR : DSLA_IMPL_SIMT;
 }
@@ -148,6 +158,10 @@ static dsla_status check_prefill_sizes(const dsla_prefill_args* a) {
     }
     if (a->impl != DSLA_IMPL_AUTO && a->impl != DSLA_IMPL_SIMT && a->impl != DSLA_IMPL_TENSOR && a->impl != DSLA_IMPL_TENSOR_PAIR)
         return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout != DSLA_GATE_SCALAR && a->gate_layout != DSLA_GATE_PER_KEY_CHANNEL) return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL) {      // the token-by-token CUDA-core kernel; chunk is ignored
+        return (a->impl == DSLA_IMPL_TENSOR || a->impl == DSLA_IMPL_TENSOR_PAIR) ? DSLA_ERR_UNSUPPORTED : DSLA_OK;
+    }
     const dsla_impl impl = resolve_impl(a);
     const int chunk = a->chunk == 0 ? 64 : a->chunk;
     if (impl == DSLA_IMPL_SIMT) {
@@ -168,7 +182,7 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     dsla_status rc = check_prefill_sizes(a);
     if (rc != DSLA_OK) return rc;
     if (!st) return DSLA_ERR_INVALID_ARG;
-    if (st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
+    if (st->n_states != 2 || st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
     if (!a->slots && a->N > st->num_slots) return DSLA_ERR_INVALID_ARG;
     if (!on_store_device(st)) return DSLA_ERR_INVALID_ARG;
     if (a->N == 0) return DSLA_OK;
@@ -191,6 +205,17 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     const int chunk = a->chunk == 0 ? 64 : a->chunk;
     p.max_chunks = (a->max_seqlen + chunk - 1) / chunk;
     p.scale = a->scale; p.use_initial_state = a->use_initial_state ? 1 : 0;
+    if (a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL) {
+        // the dual state as two states whose weights the kernel derives from gamma: (gamma, 1 - gamma)
+        RecurrentParams r{};
+        r.q = a->q; r.k = a->k; r.v = a->v; r.o = a->o;
+        r.weights = nullptr; r.cu_seqlens = a->cu_seqlens; r.slots = a->slots; r.state = st->data;
+        r.N = a->N; r.T = a->T; r.H = a->H; r.num_slots = st->num_slots; r.n_states_total = 2;
+        r.per_channel = 1; r.use_initial_state = a->use_initial_state ? 1 : 0; r.scale = a->scale;
+        r.gamma = a->gamma;
+        const float* gates[2] = {a->g_hist, a->g_rec};
+        return launch_prefill_recurrent(r, gates, 2, a->d_k, a->dtype, s);
+    }
     const dsla_impl impl = resolve_impl(a);
     if (impl != DSLA_IMPL_SIMT) return launch_prefill_tc(p, a, impl == DSLA_IMPL_TENSOR_PAIR, s);
     return launch_prefill_simt(p, a->d_k, chunk, a->dtype, s);
@@ -212,9 +237,10 @@ static dsla_status check_decode(const dsla_decode_args* a, dsla_state* st) {
     if (a->B < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0) return DSLA_ERR_INVALID_ARG;
     if (a->dtype != DSLA_F32 && a->dtype != DSLA_BF16) return DSLA_ERR_INVALID_ARG;
     if (!supported_d(a->d_k, a->d_v)) return DSLA_ERR_UNSUPPORTED;
-    if (st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
+    if (st->n_states != 2 || st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
     if (!a->slots && a->B > st->num_slots) return DSLA_ERR_INVALID_ARG;
     if (!(a->scale == a->scale)) return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout != DSLA_GATE_SCALAR && a->gate_layout != DSLA_GATE_PER_KEY_CHANNEL) return DSLA_ERR_INVALID_ARG;
     if (!on_store_device(st)) return DSLA_ERR_INVALID_ARG;
     return DSLA_OK;
 }
@@ -227,9 +253,62 @@ static dsla_status decode_device(const dsla_decode_args* a, dsla_state* st, cuda
     if (!aligned(a->q, 16) || !aligned(a->k, 16) || !aligned(a->v, 16) || !aligned(a->o, 16)) return DSLA_ERR_INVALID_ARG;
     DecodeParams p{};
     p.q = a->q; p.k = a->k; p.v = a->v; p.o = a->o;
-    p.g_hist = a->g_hist; p.g_rec = a->g_rec; p.gamma = a->gamma; p.slots = a->slots;
+    p.g[0] = a->g_hist; p.g[1] = a->g_rec; p.gamma = a->gamma; p.weights = nullptr; p.slots = a->slots;
+    p.row_mask = a->row_mask; p.n_states = 2; p.per_channel = a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL;
     p.state = st->data; p.B = a->B; p.H = a->H; p.num_slots = st->num_slots; p.scale = a->scale;
     return launch_decode(p, a->d_k, a->dtype, s);
+}
+
+// ---- n states -----------------------------------------------------------------------------
+dsla_status dsla_nstate_decode_step(const dsla_nstate_decode_args* a, dsla_state* st, void* cuda_stream) {
+    if (!a || !st) return DSLA_ERR_INVALID_ARG;
+    if (a->B < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0 || a->n_states <= 0) return DSLA_ERR_INVALID_ARG;
+    if (a->dtype != DSLA_F32 && a->dtype != DSLA_BF16) return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout != DSLA_GATE_SCALAR && a->gate_layout != DSLA_GATE_PER_KEY_CHANNEL) return DSLA_ERR_INVALID_ARG;
+    if (!supported_d(a->d_k, a->d_v) || !supported_n(a->n_states)) return DSLA_ERR_UNSUPPORTED;
+    if (st->n_states != a->n_states || st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
+    if (!a->slots && a->B > st->num_slots) return DSLA_ERR_INVALID_ARG;
+    if (!(a->scale == a->scale) || !on_store_device(st)) return DSLA_ERR_INVALID_ARG;
+    if (a->B == 0) return DSLA_OK;
+    if (!a->q || !a->k || !a->v || !a->o || !a->gates || !a->weights) return DSLA_ERR_INVALID_ARG;
+    if (!aligned(a->q, 16) || !aligned(a->k, 16) || !aligned(a->v, 16) || !aligned(a->o, 16)) return DSLA_ERR_INVALID_ARG;
+    DecodeParams p{};
+    p.q = a->q; p.k = a->k; p.v = a->v; p.o = a->o;
+    const bool pc = a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL;
+    const size_t gstride = (size_t)a->B * a->H * (pc ? a->d_k : 1);
+    for (int i = 0; i < a->n_states; ++i) p.g[i] = a->gates + (size_t)i * gstride;
+    p.gamma = nullptr; p.weights = a->weights; p.slots = a->slots; p.row_mask = a->row_mask;
+    p.n_states = a->n_states; p.per_channel = pc ? 1 : 0;
+    p.state = st->data; p.B = a->B; p.H = a->H; p.num_slots = st->num_slots; p.scale = a->scale;
+    return launch_decode(p, a->d_k, a->dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+
+dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* st, void* cuda_stream) {
+    if (!a || !st) return DSLA_ERR_INVALID_ARG;
+    if (a->N < 0 || a->T_total < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0 || a->n_states <= 0) return DSLA_ERR_INVALID_ARG;
+    if (a->dtype != DSLA_F32 && a->dtype != DSLA_BF16) return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout != DSLA_GATE_SCALAR && a->gate_layout != DSLA_GATE_PER_KEY_CHANNEL) return DSLA_ERR_INVALID_ARG;
+    if (!supported_d(a->d_k, a->d_v) || !supported_n(a->n_states)) return DSLA_ERR_UNSUPPORTED;
+    if (!a->cu_seqlens && (a->T < 0 || (long long)a->N * a->T != a->T_total)) return DSLA_ERR_INVALID_ARG;
+    if (st->n_states != a->n_states || st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
+    if (!a->slots && a->N > st->num_slots) return DSLA_ERR_INVALID_ARG;
+    if (!(a->scale == a->scale) || !on_store_device(st)) return DSLA_ERR_INVALID_ARG;
+    if (a->N == 0) return DSLA_OK;
+    if (!a->weights) return DSLA_ERR_INVALID_ARG;
+    if (a->T_total > 0) {
+        if (!a->q || !a->k || !a->v || !a->o || !a->gates) return DSLA_ERR_INVALID_ARG;
+        if (!aligned(a->q, 16) || !aligned(a->k, 16) || !aligned(a->v, 16) || !aligned(a->o, 16)) return DSLA_ERR_INVALID_ARG;
+    }
+    RecurrentParams r{};
+    r.q = a->q; r.k = a->k; r.v = a->v; r.o = a->o;
+    r.weights = a->weights; r.gamma = nullptr; r.cu_seqlens = a->cu_seqlens; r.slots = a->slots; r.state = st->data;
+    r.N = a->N; r.T = a->T; r.H = a->H; r.num_slots = st->num_slots; r.n_states_total = a->n_states;
+    const bool pc = a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL;
+    r.per_channel = pc ? 1 : 0; r.use_initial_state = a->use_initial_state ? 1 : 0; r.scale = a->scale;
+    const size_t gstride = (size_t)a->T_total * a->H * (pc ? a->d_k : 1);
+    const float* gates[8];
+    for (int i = 0; i < a->n_states; ++i) gates[i] = a->gates + (size_t)i * gstride;
+    return launch_prefill_recurrent(r, gates, a->n_states, a->d_k, a->dtype, static_cast<cudaStream_t>(cuda_stream));
 }
 
 dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cuda_stream) {
@@ -332,6 +411,7 @@ dsla_status dsla_prefill_host(const dsla_prefill_args* a, dsla_state* st, void* 
     const size_t need = dsla_prefill_staging_bytes(a);
     if (!staging || staging_bytes < need || !aligned(staging, 256)) return DSLA_ERR_INVALID_ARG;
     if (!a->q || !a->k || !a->v || !a->o || !a->g_hist || !a->g_rec) return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout != DSLA_GATE_SCALAR) return DSLA_ERR_UNSUPPORTED;      // host-buffer variants stage scalar gates only
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t tb = (size_t)a->T_total * a->H * a->d_k * esize(a->dtype), t = up256(tb);
     const size_t gb = (size_t)a->T_total * a->H * sizeof(float), g = up256(gb);
@@ -366,6 +446,7 @@ dsla_status dsla_decode_step_host(const dsla_decode_args* a, dsla_state* st, voi
     const size_t need = dsla_decode_staging_bytes(a);
     if (!staging || staging_bytes < need || !aligned(staging, 256)) return DSLA_ERR_INVALID_ARG;
     if (!a->q || !a->k || !a->v || !a->o || !a->g_hist || !a->g_rec) return DSLA_ERR_INVALID_ARG;
+    if (a->gate_layout != DSLA_GATE_SCALAR || a->row_mask) return DSLA_ERR_UNSUPPORTED;      // host-buffer variant: scalar gates, every row
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const size_t tb = (size_t)a->B * a->H * a->d_k * esize(a->dtype), t = up256(tb);
     const size_t gb = (size_t)a->B * a->H * sizeof(float), g = up256(gb);

@@ -7,9 +7,9 @@
 #include "dsla.h"
 
 struct dsla_state {
-    float* data;          // [num_slots][2][H][d_k][d_v]
+    float* data;          // [num_slots][n_states][H][d_k][d_v]
     int* status;          // device status word (0 = ok)
-    int num_slots, H, d_k, d_v;
+    int num_slots, n_states, H, d_k, d_v;
     int owns_data;
     int device;
 };
@@ -34,10 +34,26 @@ struct PrefillParams {
 struct DecodeParams {
     const void *q, *k, *v;
     void* o;
-    const float *g_hist, *g_rec, *gamma;
+    const float* g[8];          // gate of every state: [B, H], or [B, H, d_k] when per_channel
+    const float* gamma;         // [H] (dual state: weights gamma, 1 - gamma) when weights == nullptr
+    const float* weights;       // [H, n_states] or nullptr
     const int32_t* slots;
-    float* state;
-    int B, H, num_slots;
+    const uint8_t* row_mask;    // [B] or nullptr: rows with 0 are left untouched
+    float* state;               // [num_slots][n_states][H][D][D]
+    int B, H, num_slots, n_states, per_channel;
+    float scale;
+};
+
+// Launch parameters of the token-by-token prefill (one group of up to four states per launch).
+struct RecurrentParams {
+    const void *q, *k, *v;
+    void* o;
+    const float* g[4];          // gates of this launch's states: [T_total, H], or [T_total, H, d_k] when per_channel
+    const float* weights;       // [H, n_states_total], or nullptr: two states weighted (gamma, 1 - gamma)
+    const float* gamma;         // [H], used when weights == nullptr
+    const int32_t *cu_seqlens, *slots;
+    float* state;               // [num_slots][n_states_total][H][D][D]
+    int N, T, H, num_slots, n_states_total, state_first, per_channel, use_initial_state, accumulate;
     float scale;
 };
 
@@ -47,6 +63,9 @@ void count_launch(int n = 1);
 dsla_status prefill_checked(const dsla_prefill_args* a, dsla_state* st, cudaStream_t s);
 // dsla_decode.cu
 dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStream_t s);
+// dsla_prefill_recurrent.cu: gates[i] is the gate tensor of state i (n_states of them)
+dsla_status launch_prefill_recurrent(const RecurrentParams& p, const float* const* gates, int n_states, int d, dsla_dtype dt,
+                                     cudaStream_t s);
 // dsla_prefill_simt.cu
 dsla_status launch_prefill_simt(const PrefillParams& p, int d, int chunk, dsla_dtype dt, cudaStream_t s);
 // dsla_prefill_summary.cu: one warp waits, with the given poll limit, on a barrier nobody arrives at
