@@ -155,12 +155,25 @@ def test_cfg1_prefill_then_decode():
     assert rel_err(S[0, 0], S_ref[0, 0]) <= 1e-4 and rel_err(S[0, 1], S_ref[0, 1]) <= 1e-4
 
 
-def test_cfg2_prefill_full():
-    """Workload 2: bf16, B=1 H=32 d=128 T=4096, chunk 64; every output and both final states."""
+def test_cfg2_prefill_full(tc_impl):
+    """Workload 2: bf16, B=1 H=32 d=128 T=4096, chunk 64; every output and both final states, for both tensor-core
+    variants.  Besides the tolerance check (max error over the tensor's max magnitude) it prints the element-wise
+    diagnostic |x - ref| / (|ref| + 1e-3 rms(ref)): its maximum and 99.9th percentile (run pytest with -s to see it)."""
+    from util import elementwise_err, large_element_err
     c = gen.CONFIGS["cfg2"]
     inp = gen.make_dense(c["seed"], 1, c["T"], c["H"], c["d"], torch.bfloat16)
-    e = check_prefill(inp, dense=True)
-    print(f"cfg2 o rel err {e:.3e}")
+    e = check_prefill(inp, dense=True, impl=tc_impl)
+    o, S = gpu_prefill(inp, impl=tc_impl, dense=True)
+    o_ref, S_ref = oracle_prefill(inp)
+    mx, p999 = elementwise_err(o, o_ref)
+    smx, sp999 = elementwise_err(S, S_ref)
+    lo, ls = large_element_err(o, o_ref), large_element_err(S, S_ref)
+    print(f"cfg2 [{tc_impl}] o: rel err {e:.3e}, element-wise max {mx:.3e}, 99.9th pct {p999:.3e}, elements >= rms {lo:.3e}; "
+          f"states: rel err {rel_err(S, S_ref):.3e}, element-wise max {smx:.3e}, 99.9th pct {sp999:.3e}, elements >= rms {ls:.3e}")
+    # The absolute error is of the order of 5e-3 of the tensor's largest magnitude whatever the element (operand roundings
+    # accumulate over the whole dot product), so elements far below the rms can be off by a multiple of themselves: the
+    # element-wise figures are reported, and bounded only where an element is at least as large as the rms.
+    assert lo <= 0.1 and ls <= 0.1
 
 
 def test_prefill_composition_on_gpu():

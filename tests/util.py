@@ -26,6 +26,14 @@ def elementwise_err(x, ref):
     return float(e.max()), float(np.quantile(e, 0.999))
 
 
+def large_element_err(x, ref):
+    """max |x - ref| / |ref| over the elements whose magnitude is at least the tensor's rms."""
+    x = np.asarray(x, dtype=np.float64).ravel()
+    ref = np.asarray(ref, dtype=np.float64).ravel()
+    big = np.abs(ref) >= np.sqrt(np.mean(ref * ref))
+    return float(np.max(np.abs(x - ref)[big] / np.abs(ref)[big])) if big.any() else 0.0
+
+
 def oracle_prefill(inp, state0=None, slots=None, scale=1.0, nthreads=None):
     from oracle import dsla_oracle as orc
     f = inp.as_f64()
