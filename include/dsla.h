@@ -257,6 +257,27 @@ typedef struct {
 dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* st, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Gate producer.  The gates of the two states come from single linear layers on the layer's input (Sec. 5.3; App. B:
+ * zero bias, history layer near identity, recency layer random at initialisation).  This entry point computes
+ *     [g_hist | g_rec][t, :] = logistic(x[t, :] W^T + bias)
+ * on the tensor cores and writes the two [T, H] fp32 tensors dsla_prefill / dsla_decode_step read, so the
+ * pre-activations never exist in memory.  Rows 0 .. H-1 of W (and of bias) produce the history gates, rows H .. 2H-1
+ * the recency gates.  Requirements: H a multiple of 8 with 2 H <= 256; D_model a multiple of 64; x, w 16-byte aligned,
+ * g_hist, g_rec 16-byte aligned; else DSLA_ERR_INVALID_ARG / DSLA_ERR_UNSUPPORTED.  dsla_gate_project_last_error reads
+ * (synchronising the device) and clears the kernel's time-out flag: DSLA_OK or DSLA_ERR_TIMEOUT.
+ * ------------------------------------------------------------------------------------------ */
+typedef struct {
+    const void* x;          /* [T, D_model] bf16, row-major                                               */
+    const void* w;          /* [2 H, D_model] bf16, row-major (one row per output)                        */
+    const float* bias;      /* [2 H] fp32 or NULL                                                         */
+    float* g_hist;          /* [T, H] fp32 (output)                                                       */
+    float* g_rec;           /* [T, H] fp32 (output)                                                       */
+    int T, H, D_model;
+} dsla_gate_project_args;
+dsla_status dsla_gate_project(const dsla_gate_project_args* a, void* cuda_stream);
+dsla_status dsla_gate_project_last_error(void);
+
+/* ------------------------------------------------------------------------------------------
  * Host-buffer variants (end-to-end path): q, k, v, o, g_hist, g_rec in `a` are HOST pointers
  * (pinned memory gives asynchronous copies); gamma, cu_seqlens, slots and the workspace stay
  * device pointers.  `staging` is caller-owned device memory of at least

@@ -47,6 +47,11 @@ class dsla_decode_args(Structure):
                 ("dtype", c_int), ("scale", c_float), ("gate_layout", c_int), ("row_mask", c_void_p)]
 
 
+class dsla_gate_project_args(Structure):
+    _fields_ = [("x", c_void_p), ("w", c_void_p), ("bias", c_void_p), ("g_hist", c_void_p), ("g_rec", c_void_p),
+                ("T", c_int), ("H", c_int), ("D_model", c_int)]
+
+
 class dsla_nstate_decode_args(Structure):
     _fields_ = [("q", c_void_p), ("k", c_void_p), ("v", c_void_p), ("o", c_void_p),
                 ("gates", c_void_p), ("weights", c_void_p), ("slots", c_void_p), ("row_mask", c_void_p),
@@ -78,6 +83,10 @@ _lib.dsla_nstate_decode_step.argtypes = [POINTER(dsla_nstate_decode_args), c_voi
 _lib.dsla_nstate_decode_step.restype = c_int
 _lib.dsla_nstate_prefill.argtypes = [POINTER(dsla_nstate_prefill_args), c_void_p, c_void_p]
 _lib.dsla_nstate_prefill.restype = c_int
+_lib.dsla_gate_project.argtypes = [POINTER(dsla_gate_project_args), c_void_p]
+_lib.dsla_gate_project.restype = c_int
+_lib.dsla_gate_project_last_error.argtypes = []
+_lib.dsla_gate_project_last_error.restype = c_int
 _lib.dsla_state_free.argtypes = [c_void_p]
 _lib.dsla_state_free.restype = c_int
 _lib.dsla_state_data.argtypes = [c_void_p]
@@ -399,3 +408,23 @@ def dsla_nstate_prefill(q, k, v, gates, weights, st: DslaState, *, o=None, cu_se
     a.gate_layout = DSLA_GATE_PER_KEY_CHANNEL if gates.dim() == 4 else DSLA_GATE_SCALAR
     _check(_lib.dsla_nstate_prefill(byref(a), st.handle, _stream(stream)), "dsla_nstate_prefill")
     return o
+
+
+def dsla_gate_project(x, w, bias=None, *, g_hist=None, g_rec=None, stream=None):
+    """logistic(x W^T + bias) on the tensor cores: x [T, D_model] bf16, w [2 H, D_model] bf16, bias [2 H] fp32 or None.
+    Returns (g_hist, g_rec), both [T, H] fp32."""
+    T, D_model = x.shape
+    H = w.shape[0] // 2
+    if g_hist is None:
+        g_hist = torch.empty((T, H), dtype=torch.float32, device=x.device)
+    if g_rec is None:
+        g_rec = torch.empty((T, H), dtype=torch.float32, device=x.device)
+    a = dsla_gate_project_args()
+    a.x, a.w, a.bias, a.g_hist, a.g_rec = _ptr(x), _ptr(w), _ptr(bias), _ptr(g_hist), _ptr(g_rec)
+    a.T, a.H, a.D_model = int(T), int(H), int(D_model)
+    _check(_lib.dsla_gate_project(byref(a), _stream(stream)), "dsla_gate_project")
+    return g_hist, g_rec
+
+
+def dsla_gate_project_last_error() -> int:
+    return int(_lib.dsla_gate_project_last_error())

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdsla.so")
-SOURCES = ["dsla_api.cu", "dsla_decode.cu", "dsla_prefill_simt.cu", "dsla_prefill_recurrent.cu", "dsla_prefill_summary.cu", "dsla_prefill_tc.cu",
+SOURCES = ["dsla_api.cu", "dsla_decode.cu", "dsla_gate_project.cu", "dsla_prefill_simt.cu", "dsla_prefill_recurrent.cu", "dsla_prefill_summary.cu", "dsla_prefill_tc.cu",
            "dsla_prefill_tc_pair.cu", "dsla_static_ws.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),

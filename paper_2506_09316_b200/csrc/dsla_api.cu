@@ -315,6 +315,18 @@ dsla_status dsla_decode_step(const dsla_decode_args* a, dsla_state* st, void* cu
     return decode_device(a, st, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---- gate producer ------------------------------------------------------------------------
+dsla_status dsla_gate_project(const dsla_gate_project_args* a, void* cuda_stream) {
+    if (!a || a->T < 0 || a->H <= 0 || a->D_model <= 0) return DSLA_ERR_INVALID_ARG;
+    if (a->H % 8 != 0 || 2 * a->H > 256 || a->D_model % 64 != 0) return DSLA_ERR_UNSUPPORTED;
+    if (a->T == 0) return DSLA_OK;
+    if (!a->x || !a->w || !a->g_hist || !a->g_rec) return DSLA_ERR_INVALID_ARG;
+    if (!aligned(a->x, 16) || !aligned(a->w, 16) || !aligned(a->g_hist, 16) || !aligned(a->g_rec, 16)) return DSLA_ERR_INVALID_ARG;
+    return launch_gate_project(a, static_cast<cudaStream_t>(cuda_stream));
+}
+
+dsla_status dsla_gate_project_last_error(void) { return gate_project_last_error(); }
+
 // ---- host-buffer variants -----------------------------------------------------------------
 static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 

@@ -63,6 +63,9 @@ void count_launch(int n = 1);
 dsla_status prefill_checked(const dsla_prefill_args* a, dsla_state* st, cudaStream_t s);
 // dsla_decode.cu
 dsla_status launch_decode(const DecodeParams& p, int d, dsla_dtype dt, cudaStream_t s);
+// dsla_gate_project.cu
+dsla_status launch_gate_project(const dsla_gate_project_args* a, cudaStream_t s);
+dsla_status gate_project_last_error();
 // dsla_prefill_recurrent.cu: gates[i] is the gate tensor of state i (n_states of them)
 dsla_status launch_prefill_recurrent(const RecurrentParams& p, const float* const* gates, int n_states, int d, dsla_dtype dt,
                                      cudaStream_t s);

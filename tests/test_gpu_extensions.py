@@ -216,3 +216,56 @@ def test_nstate_entry_points_check_the_store():
     with pytest.raises(dsla.DslaError) as e:            # three states: no kernel
         dsla.dsla_state_alloc_n(2, 3, 2, 64, 64)
     assert e.value.status == dsla.DSLA_ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------------------------------ gate producer
+@pytest.mark.parametrize("T,H,D_model,with_bias", [(1, 8, 64, False), (130, 32, 512, True), (4096, 32, 4096, False),
+                                                   (300, 16, 1024, True), (257, 128, 256, True)])
+def test_gate_project(T, H, D_model, with_bias):
+    """logistic(x W^T + b) against the fp64 checker (bf16 inputs widened exactly; products are exact in fp32, so only the
+    summation order, the fp32 accumulator and the approximate exponential differ), then straight into a prefill."""
+    import paper_2506_09316_b200 as dsla
+    rng = np.random.default_rng(3900 + T)
+    x = torch.from_numpy(rng.normal(size=(T, D_model)).astype(np.float32)).to(BF)
+    w = torch.from_numpy((rng.normal(size=(2 * H, D_model)) * (2.0 / np.sqrt(D_model))).astype(np.float32)).to(BF)
+    b = torch.from_numpy(rng.normal(size=2 * H).astype(np.float32) * 2.0) if with_bias else None
+    gh = torch.full((T, H), float("nan"), device="cuda")
+    gr = torch.full((T, H), float("nan"), device="cuda")
+    dsla.dsla_gate_project(x.cuda(), w.cuda(), None if b is None else b.cuda(), g_hist=gh, g_rec=gr)
+    torch.cuda.synchronize()
+    assert dsla.dsla_gate_project_last_error() == dsla.DSLA_OK
+    ref = orc.gate_project(x.double().numpy(), w.double().numpy().T, None if b is None else b.double().numpy())
+    got = np.concatenate([_f64(gh), _f64(gr)], axis=1)
+    assert np.max(np.abs(got - ref)) <= 2e-5, np.max(np.abs(got - ref))
+    assert got.min() >= 0.0 and got.max() <= 1.0
+
+
+def test_gate_project_feeds_the_prefill():
+    import paper_2506_09316_b200 as dsla
+    rng = np.random.default_rng(3950)
+    T, H, d, D_model = 300, 8, 128, 256
+    inp = gen.make_dense(3951, 1, T, H, d, BF)
+    x = torch.from_numpy(rng.normal(size=(T, D_model)).astype(np.float32)).to(BF)
+    w = torch.from_numpy((rng.normal(size=(2 * H, D_model)) / np.sqrt(D_model)).astype(np.float32)).to(BF)
+    b = torch.from_numpy(np.concatenate([np.full(H, 5.0), np.full(H, 1.0)]).astype(np.float32))
+    gh, gr = dsla.dsla_gate_project(x.cuda(), w.cuda(), b.cuda())
+    dv = inp.to("cuda")
+    st = dsla.dsla_state_alloc(1, H, d, d)
+    o = dsla.dsla_prefill(dv.q, dv.k, dv.v, gh, gr, dv.gamma, st, max_seqlen=T)
+    torch.cuda.synchronize()
+    g = orc.gate_project(x.double().numpy(), w.double().numpy().T, b.double().numpy())
+    f = inp.as_f64()
+    o_ref, S_ref = orc.prefill(f["q"], f["k"], f["v"], g[:, :H], g[:, H:], f["gamma"])
+    assert rel_err(_f64(o), o_ref) <= TOL[BF] and rel_err(_f64(st.tensor), S_ref) <= TOL[BF]
+
+
+def test_gate_project_rejects_unsupported_shapes():
+    import paper_2506_09316_b200 as dsla
+    x = torch.zeros(4, 100, dtype=BF, device="cuda")
+    w = torch.zeros(16, 100, dtype=BF, device="cuda")
+    with pytest.raises(dsla.DslaError) as e:
+        dsla.dsla_gate_project(x, w)                       # D_model not a multiple of 64
+    assert e.value.status == dsla.DSLA_ERR_UNSUPPORTED
+    with pytest.raises(dsla.DslaError) as e:
+        dsla.dsla_gate_project(torch.zeros(4, 128, dtype=BF, device="cuda"), torch.zeros(12, 128, dtype=BF, device="cuda"))   # H = 6
+    assert e.value.status == dsla.DSLA_ERR_UNSUPPORTED
