@@ -141,6 +141,7 @@ KERNEL_SOURCES = {   # the files whose change makes a stored DRAM-traffic figure
     "tensor": ["dsla_prefill_tc.cu", "dsla_prefill_summary.cu", "dsla_prefill_tc.cuh", "tc_utils.cuh"],
     "pair": ["dsla_prefill_tc_pair.cu", "dsla_prefill_summary.cu", "dsla_prefill_tc.cuh", "tc_utils.cuh"],
     "decode": ["dsla_decode.cu"],
+    "gate": ["dsla_gate_project.cu", "tc_utils.cuh"],
 }
 
 
@@ -340,6 +341,10 @@ def bench_ours(args):
         if not args.no_more:
             decode["n_states"] = bench_decode_nstate(dsla, peaks, dev, rank)
 
+    gate_producer = None
+    if not args.no_gate:
+        gate_producer = bench_gate_project(dsla, peaks, dev, rank)
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu_baseline = time_oracle_sample(spec, lens, budget_s=args.cpu_seconds)
@@ -356,7 +361,7 @@ def bench_ours(args):
             "prefill_only": {"value": world * T_total / (prefill_ms * 1e-3), "unit": "tokens/s (one layer)", "ms": prefill_ms},
             "decode_leg_ms": decode_leg_ms,
             "roofline": roofline, "prefill_sustained": sustained, "prefill_more": more, "decode": decode,
-            "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gate_producer": gate_producer, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
         }
         print(json.dumps(line))
@@ -494,6 +499,41 @@ def bench_decode_nstate(dsla, peaks, dev, rank):
 
 
 # --------------------------------------------------------------------------------------------
+def bench_gate_project(dsla, peaks, dev, rank):
+    """The gate producer (logistic(x W^T + b) on the tensor cores) for the tokens of one prefill: HBM-bound on reading x once.
+    Input sets rotate so that x comes from DRAM (the sets together exceed L2)."""
+    out = {}
+    H, D_model = 32, 4096
+    for name, T in (("T4096", 4096), ("T65536", 65536)):
+        n_sets = max(2, int(np.ceil(160e6 / (T * D_model * 2))) + 1)
+        g = torch.Generator(device=dev).manual_seed(4200 + rank)
+        xs = [torch.randn((T, D_model), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16) for _ in range(n_sets)]
+        w = (torch.randn((2 * H, D_model), generator=g, device=dev, dtype=torch.float32) / 64.0).to(torch.bfloat16)
+        b = torch.zeros(2 * H, device=dev, dtype=torch.float32)
+        gh = torch.empty((T, H), device=dev, dtype=torch.float32)
+        gr = torch.empty((T, H), device=dev, dtype=torch.float32)
+        for i in range(3):
+            dsla.dsla_gate_project(xs[i % n_sets], w, b, g_hist=gh, g_rec=gr)
+        torch.cuda.synchronize()
+        steps = 20
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for i in range(steps):
+            evs[i][0].record()
+            dsla.dsla_gate_project(xs[i % n_sets], w, b, g_hist=gh, g_rec=gr)
+            evs[i][1].record()
+        torch.cuda.synchronize()
+        ms = [e[0].elapsed_time(e[1]) for e in evs]
+        nbytes = T * D_model * 2 + 2 * H * D_model * 2 + 2 * T * H * 4
+        med = float(np.median(ms))
+        out[name] = {"T": T, "H": H, "D_model": D_model, "ctas": (T + 127) // 128, "median_us": med * 1e3, "best_us": float(np.min(ms)) * 1e3,
+                     "algorithmic_bytes": nbytes, "achieved_gbs": nbytes / (med * 1e-3) / 1e9,
+                     "frac_of_hbm_peak": nbytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": stored_traffic("gate", name),
+                     "tflops": 2.0 * T * 2 * H * D_model / (med * 1e-3) / 1e12}
+        del xs
+        torch.cuda.empty_cache()
+    return out
+
+
 def time_oracle_sample(spec, lens, budget_s=15.0):
     """Times the CPU checker, as it stands, on a bounded sample of the same workload: the first
     `heads` heads of the first sequences, all their tokens (units are independent)."""
@@ -562,6 +602,7 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=0.6)
     ap.add_argument("--no-sustained", action="store_true")
     ap.add_argument("--no-more", action="store_true", help="skip the further prefill workloads and the n-state decode section")
+    ap.add_argument("--no-gate", action="store_true", help="skip the gate-producer section")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
