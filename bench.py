@@ -341,6 +341,10 @@ def bench_ours(args):
         if not args.no_more:
             decode["n_states"] = bench_decode_nstate(dsla, peaks, dev, rank)
 
+    extensions = None
+    if not args.no_more and not args.no_decode:
+        extensions = bench_extensions(dsla, peaks, dev, rank)
+
     gate_producer = None
     if not args.no_gate:
         gate_producer = bench_gate_project(dsla, peaks, dev, rank)
@@ -361,7 +365,7 @@ def bench_ours(args):
             "prefill_only": {"value": world * T_total / (prefill_ms * 1e-3), "unit": "tokens/s (one layer)", "ms": prefill_ms},
             "decode_leg_ms": decode_leg_ms,
             "roofline": roofline, "prefill_sustained": sustained, "prefill_more": more, "decode": decode,
-            "gate_producer": gate_producer, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gate_producer": gate_producer, "extensions": extensions, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
         }
         print(json.dumps(line))
@@ -499,6 +503,84 @@ def bench_decode_nstate(dsla, peaks, dev, rank):
 
 
 # --------------------------------------------------------------------------------------------
+def bench_extensions(dsla, peaks, dev, rank):
+    """The wider forms of the layer: gates per key channel (decode and prefill), a decode batch in which half of the rows
+    belong to another layer type (row mask), n-state prefill.  Decode sections: B=128, H=32, d=128, a stack of layers whose
+    states total about 4 GB (>> L2); prefill sections: the cfg2 shape (one sequence of 4096 tokens, 32 heads)."""
+    c = gen.CONFIGS["cfg4"]
+    B, H, d = c["B"], c["H"], c["d"]
+    out = {}
+    L = 7
+    g = torch.Generator(device=dev)
+    g.manual_seed(c["seed"] + 900 + rank)
+    states = [dsla.dsla_state_alloc(B, H, d, d, device=dev) for _ in range(L)]
+    for s_ in states:
+        s_.tensor.normal_(0.0, c["state_std"], generator=g)
+    inp = gen.make_packed_device(c["seed"] + 901 + rank, [1] * (L * B), H, d, torch.bfloat16, device=dev)
+    view = lambda t: t.view(L, B, *t.shape[1:])
+    q, k, v, gs1, gs2 = map(view, (inp.q, inp.k, inp.v, inp.g_hist, inp.g_rec))
+    gv1 = torch.sigmoid(torch.randn((L, B, H, d), generator=g, device=dev) * 0.5 + 6.0)
+    gv2 = torch.sigmoid(torch.randn((L, B, H, d), generator=g, device=dev) * 0.5 + 1.0)
+    mask = (torch.arange(B, device=dev) % 2 == 0).to(torch.uint8)
+    o = torch.empty_like(v)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, steps=32):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / steps
+
+    def per_channel():
+        for l in range(L):
+            dsla.dsla_decode_step(q[l], k[l], v[l], gv1[l], gv2[l], inp.gamma, states[l], o=o[l])
+
+    def masked():
+        for l in range(L):
+            dsla.dsla_decode_step(q[l], k[l], v[l], gs1[l], gs2[l], inp.gamma, states[l], o=o[l], row_mask=mask)
+
+    t = timed(per_channel) / L
+    nbytes = B * H * (4 * d * d * 4 + 4 * d * 2 + 2 * d * 4)
+    out["decode_per_key_channel_gates"] = {"layers": L, "us_per_launch": t * 1e6, "algorithmic_bytes": nbytes, "achieved": nbytes / t / 1e9,
+                                           "unit": "GB/s", "frac": nbytes / t / 1e9 / peaks["hbm_gbs"]}
+    t = timed(masked) / L
+    nbytes = (B // 2) * H * DECODE_BYTES_PER_ROW_HEAD(d, 2)
+    out["decode_row_mask_half"] = {"layers": L, "us_per_launch": t * 1e6, "algorithmic_bytes": nbytes, "achieved": nbytes / t / 1e9,
+                                   "unit": "GB/s", "frac": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                                   "note": "every other row masked: only the live rows' states move"}
+    del states, inp, q, k, v, gs1, gs2, gv1, gv2, o
+    torch.cuda.empty_cache()
+
+    T = 4096
+    pin = gen.make_packed_device(c["seed"] + 902 + rank, [T], H, d, torch.bfloat16, device=dev)
+    st = dsla.dsla_state_alloc(1, H, d, d, device=dev)
+    gc1 = torch.sigmoid(torch.randn((T, H, d), generator=g, device=dev) * 0.5 + 6.0)
+    gc2 = torch.sigmoid(torch.randn((T, H, d), generator=g, device=dev) * 0.5 + 1.0)
+    oo = torch.empty_like(pin.v)
+    t = timed(lambda: dsla.dsla_prefill(pin.q, pin.k, pin.v, gc1, gc2, pin.gamma, st, o=oo, max_seqlen=T), steps=5)
+    out["prefill_per_key_channel_gates"] = {"workload": f"N=1 H={H} d={d} T={T} bf16", "ms": t * 1e3, "tokens_per_s": T / t,
+                                            "kernel": "token-by-token CUDA-core recurrence"}
+    for n in (2, 4):
+        stn = dsla.dsla_state_alloc_n(1, n, H, d, d, device=dev)
+        gates = torch.sigmoid(torch.randn((n, T, H), generator=g, device=dev) * 0.5 + 3.0)
+        w = torch.rand((H, n), generator=g, device=dev)
+        ws = torch.empty(max(1, dsla.dsla_nstate_prefill_workspace_bytes(pin.q, pin.k, pin.v, gates, w, max_seqlen=T)), dtype=torch.uint8, device=dev)
+        t = timed(lambda: dsla.dsla_nstate_prefill(pin.q, pin.k, pin.v, gates, w, stn, o=oo, max_seqlen=T, workspace=ws), steps=10)
+        t2 = timed(lambda: dsla.dsla_nstate_prefill(pin.q, pin.k, pin.v, gates, w, stn, o=oo, max_seqlen=T, impl="simt"), steps=3)
+        flops = T * H * (2 * 64 * 2 * d + n * 4 * d * d) * (n // 2) / max(n // 2, 1) if n < 2 else T * H * (n // 2) * FLOP_PER_TOKEN_HEAD(d, 64)
+        out[f"prefill_{n}_states"] = {"workload": f"N=1 H={H} d={d} T={T} bf16, scalar gates", "ms": t * 1e3, "tokens_per_s": T / t,
+                                      "kernel": f"chunkwise tensor-core kernel, {n // 2} pass(es) of two states",
+                                      "executed_tflops": flops / t / 1e12, "token_by_token_kernel_ms": t2 * 1e3}
+        del stn, ws
+    return out
+
+
 def bench_gate_project(dsla, peaks, dev, rank):
     """The gate producer (logistic(x W^T + b) on the tensor cores) for the tokens of one prefill: HBM-bound on reading x once.
     Input sets rotate so that x comes from DRAM (the sets together exceed L2)."""

@@ -249,11 +249,22 @@ typedef struct {
     float scale;
     int use_initial_state;
     dsla_gate_layout gate_layout;
+    int max_seqlen;             /* as in dsla_prefill_args (dense batches: T)                                  */
+    dsla_impl impl;             /* AUTO, SIMT (the token-by-token kernel) or TENSOR                           */
+    void* workspace;            /* device scratch of dsla_nstate_prefill_workspace_bytes(a) bytes, 256-byte    */
+    size_t workspace_bytes;     /* aligned; may be NULL / 0 when that function returns 0                       */
 } dsla_nstate_prefill_args;
 
-/* Prefill of the n-state form on CUDA cores, token by token (fp32 arithmetic, no workspace).  With more than four
- * states (more than two when the gates are per key channel and d = 128) the states are processed in groups, each group
- * adding its share to o, so o is rounded to dtype once per group. */
+/* Prefill of the n-state form.  Two kernels:
+ *  - SIMT: the recurrence itself on CUDA cores, token by token (fp32 arithmetic, no workspace), for every supported
+ *    n, dtype, d and gate layout.  With more than four states (more than two when the gates are per key channel and
+ *    d = 128) the states are processed in groups, each group adding its share to o.
+ *  - TENSOR (what AUTO picks when it applies): bf16, d = 128, scalar gates, n in {2, 4, 8}: the chunkwise tensor-core
+ *    kernel of dsla_prefill run once per pair of states (2i, 2i + 1) with the weights (w_2i, w_2i+1); pairs after the
+ *    first write their share to a scratch tensor in the workspace that is then added to o, so o is rounded to bf16 once
+ *    per pair.  Needs the workspace below.
+ * Errors as dsla_prefill; time-outs and a too small max_seqlen are reported through dsla_state_last_error. */
+size_t dsla_nstate_prefill_workspace_bytes(const dsla_nstate_prefill_args* a);
 dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* st, void* cuda_stream);
 
 /* ------------------------------------------------------------------------------------------

@@ -64,7 +64,8 @@ class dsla_nstate_prefill_args(Structure):
                 ("gates", c_void_p), ("weights", c_void_p), ("cu_seqlens", c_void_p), ("slots", c_void_p),
                 ("N", c_int), ("T", c_int), ("T_total", c_int), ("H", c_int), ("d_k", c_int), ("d_v", c_int),
                 ("n_states", c_int), ("dtype", c_int), ("scale", c_float), ("use_initial_state", c_int),
-                ("gate_layout", c_int)]
+                ("gate_layout", c_int), ("max_seqlen", c_int), ("impl", c_int), ("workspace", c_void_p),
+                ("workspace_bytes", c_size_t)]
 
 
 _lib.dsla_status_string.argtypes = [c_int]
@@ -83,6 +84,8 @@ _lib.dsla_nstate_decode_step.argtypes = [POINTER(dsla_nstate_decode_args), c_voi
 _lib.dsla_nstate_decode_step.restype = c_int
 _lib.dsla_nstate_prefill.argtypes = [POINTER(dsla_nstate_prefill_args), c_void_p, c_void_p]
 _lib.dsla_nstate_prefill.restype = c_int
+_lib.dsla_nstate_prefill_workspace_bytes.argtypes = [POINTER(dsla_nstate_prefill_args)]
+_lib.dsla_nstate_prefill_workspace_bytes.restype = c_size_t
 _lib.dsla_gate_project.argtypes = [POINTER(dsla_gate_project_args), c_void_p]
 _lib.dsla_gate_project.restype = c_int
 _lib.dsla_gate_project_last_error.argtypes = []
@@ -386,17 +389,16 @@ def dsla_nstate_decode_step(q, k, v, gates, weights, st: DslaState, *, o=None, s
     return o
 
 
-def dsla_nstate_prefill(q, k, v, gates, weights, st: DslaState, *, o=None, cu_seqlens=None, slots=None, max_seqlen=None,
-                        scale=1.0, use_initial_state=False, stream=None):
-    """n-state prefill (CUDA cores, token by token): gates [n, T_total, H] (or [n, T_total, H, d]), weights [H, n]."""
+def _nstate_prefill_args(q, k, v, o, gates, weights, cu_seqlens, slots, max_seqlen, scale, use_initial_state, impl):
     T_total, H, d_k = q.shape
     if cu_seqlens is None:
         T = int(max_seqlen) if max_seqlen is not None else T_total
         N = T_total // T if T > 0 else 0
+        max_seqlen = T
     else:
         N, T = cu_seqlens.numel() - 1, 0
-    if o is None:
-        o = torch.empty_like(v)
+        if max_seqlen is None:
+            max_seqlen = T_total      # an upper bound is valid (the tighter the bound, the better the segment plan)
     a = dsla_nstate_prefill_args()
     a.q, a.k, a.v, a.o = _ptr(q), _ptr(k), _ptr(v), _ptr(o)
     a.gates, a.weights, a.cu_seqlens, a.slots = _ptr(gates), _ptr(weights), _ptr(cu_seqlens), _ptr(slots)
@@ -406,6 +408,31 @@ def dsla_nstate_prefill(q, k, v, gates, weights, st: DslaState, *, o=None, cu_se
     a.scale = float(scale)
     a.use_initial_state = int(bool(use_initial_state))
     a.gate_layout = DSLA_GATE_PER_KEY_CHANNEL if gates.dim() == 4 else DSLA_GATE_SCALAR
+    a.max_seqlen = int(max_seqlen)
+    a.impl = _IMPLS[impl]
+    return a
+
+
+def dsla_nstate_prefill_workspace_bytes(q, k, v, gates, weights, *, cu_seqlens=None, max_seqlen=None, impl="auto") -> int:
+    """Scratch bytes ``dsla_nstate_prefill`` needs for these tensors (0 for the token-by-token kernel)."""
+    a = _nstate_prefill_args(q, k, v, v, gates, weights, cu_seqlens, None, max_seqlen, 1.0, False, impl)
+    return int(_lib.dsla_nstate_prefill_workspace_bytes(byref(a)))
+
+
+def dsla_nstate_prefill(q, k, v, gates, weights, st: DslaState, *, o=None, cu_seqlens=None, slots=None, max_seqlen=None,
+                        scale=1.0, use_initial_state=False, impl="auto", workspace=None, stream=None):
+    """n-state prefill: gates [n, T_total, H] (or [n, T_total, H, d] per key channel), weights [H, n].  bf16, d = 128,
+    scalar gates and an even n run on the chunkwise tensor-core kernel, one pass per pair of states (``impl="simt"``
+    forces the token-by-token CUDA-core kernel, which serves everything else)."""
+    if o is None:
+        o = torch.empty_like(v)
+    a = _nstate_prefill_args(q, k, v, o, gates, weights, cu_seqlens, slots, max_seqlen, scale, use_initial_state, impl)
+    if workspace is None:
+        need = int(_lib.dsla_nstate_prefill_workspace_bytes(byref(a)))
+        if need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    a.workspace = _ptr(workspace)
+    a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(_lib.dsla_nstate_prefill(byref(a), st.handle, _stream(stream)), "dsla_nstate_prefill")
     return o
 

@@ -19,6 +19,22 @@ __global__ void zero_slots_kernel(float* data, const int32_t* slots, int num_slo
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x)
         base[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 }
+
+// o += t over n8 pieces of eight bf16 (fp32 sum, one rounding): the share of a later pair of states of the n-state prefill
+__global__ void __launch_bounds__(256) add_bf16_kernel(uint4* __restrict__ o, const uint4* __restrict__ t, size_t n8) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+        uint4 a = o[i];
+        const uint4 b = __ldcs(t + i);
+        __nv_bfloat162* pa = reinterpret_cast<__nv_bfloat162*>(&a);
+        const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 x = __bfloat1622float2(pa[e]), y = __bfloat1622float2(pb[e]);
+            pa[e] = __floats2bfloat162_rn(x.x + y.x, x.y + y.y);
+        }
+        o[i] = a;
+    }
+}
 }  // namespace dsla
 
 using namespace dsla;
@@ -205,6 +221,7 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     const int chunk = a->chunk == 0 ? 64 : a->chunk;
     p.max_chunks = (a->max_seqlen + chunk - 1) / chunk;
     p.scale = a->scale; p.use_initial_state = a->use_initial_state ? 1 : 0;
+    p.weights = nullptr; p.n_total = 2; p.state_first = 0;
     if (a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL) {
         // the dual state as two states whose weights the kernel derives from gamma: (gamma, 1 - gamma)
         RecurrentParams r{};
@@ -283,13 +300,54 @@ dsla_status dsla_nstate_decode_step(const dsla_nstate_decode_args* a, dsla_state
     return launch_decode(p, a->d_k, a->dtype, static_cast<cudaStream_t>(cuda_stream));
 }
 
-dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* st, void* cuda_stream) {
-    if (!a || !st) return DSLA_ERR_INVALID_ARG;
-    if (a->N < 0 || a->T_total < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0 || a->n_states <= 0) return DSLA_ERR_INVALID_ARG;
+// the n-state prefill as a dual-state prefill problem of the same sizes (what the segment plan and the workspace depend on)
+static dsla_prefill_args nstate_as_prefill_args(const dsla_nstate_prefill_args* a) {
+    dsla_prefill_args b{};
+    b.q = a->q; b.k = a->k; b.v = a->v; b.o = a->o;
+    b.cu_seqlens = a->cu_seqlens; b.slots = a->slots;
+    b.N = a->N; b.T = a->T; b.T_total = a->T_total; b.max_seqlen = a->max_seqlen; b.H = a->H; b.d_k = a->d_k; b.d_v = a->d_v;
+    b.chunk = 64; b.dtype = a->dtype; b.scale = a->scale; b.use_initial_state = a->use_initial_state;
+    b.impl = DSLA_IMPL_TENSOR; b.gate_layout = DSLA_GATE_SCALAR;
+    b.workspace = a->workspace; b.workspace_bytes = a->workspace_bytes;
+    return b;
+}
+
+static dsla_status check_nstate_prefill_sizes(const dsla_nstate_prefill_args* a) {
+    if (!a) return DSLA_ERR_INVALID_ARG;
+    if (a->N < 0 || a->T_total < 0 || a->H <= 0 || a->d_k <= 0 || a->d_v <= 0 || a->n_states <= 0 || a->max_seqlen < 0) return DSLA_ERR_INVALID_ARG;
     if (a->dtype != DSLA_F32 && a->dtype != DSLA_BF16) return DSLA_ERR_INVALID_ARG;
     if (a->gate_layout != DSLA_GATE_SCALAR && a->gate_layout != DSLA_GATE_PER_KEY_CHANNEL) return DSLA_ERR_INVALID_ARG;
+    if (a->impl != DSLA_IMPL_AUTO && a->impl != DSLA_IMPL_SIMT && a->impl != DSLA_IMPL_TENSOR) return DSLA_ERR_INVALID_ARG;
     if (!supported_d(a->d_k, a->d_v) || !supported_n(a->n_states)) return DSLA_ERR_UNSUPPORTED;
-    if (!a->cu_seqlens && (a->T < 0 || (long long)a->N * a->T != a->T_total)) return DSLA_ERR_INVALID_ARG;
+    if (!a->cu_seqlens) {
+        if (a->T < 0 || (long long)a->N * a->T != a->T_total || a->max_seqlen < a->T) return DSLA_ERR_INVALID_ARG;
+    } else if (a->max_seqlen > a->T_total) {
+        return DSLA_ERR_INVALID_ARG;
+    }
+    return DSLA_OK;
+}
+
+// pairs of states through the chunkwise tensor-core kernel: bf16, d = 128, scalar gates, an even number of states
+static bool nstate_tensor_applies(const dsla_nstate_prefill_args* a) {
+    return a->dtype == DSLA_BF16 && a->d_k == 128 && a->gate_layout == DSLA_GATE_SCALAR && a->n_states % 2 == 0 && prefill_tc_available();
+}
+
+// pairs after the first write their share of o to a scratch tensor that is then added to o
+static size_t nstate_o_scratch_bytes(const dsla_nstate_prefill_args* a) {
+    return a->n_states > 2 ? (((size_t)a->T_total * a->H * a->d_v * 2 + 255) & ~(size_t)255) : 0;
+}
+
+size_t dsla_nstate_prefill_workspace_bytes(const dsla_nstate_prefill_args* a) {
+    if (check_nstate_prefill_sizes(a) != DSLA_OK || a->impl == DSLA_IMPL_SIMT || !nstate_tensor_applies(a)) return 0;
+    const dsla_prefill_args b = nstate_as_prefill_args(a);
+    return prefill_tc_workspace_bytes(&b, false) + nstate_o_scratch_bytes(a);
+}
+
+dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* st, void* cuda_stream) {
+    if (!a || !st) return DSLA_ERR_INVALID_ARG;
+    const dsla_status rc0 = check_nstate_prefill_sizes(a);
+    if (rc0 != DSLA_OK) return rc0;
+    if (a->impl == DSLA_IMPL_TENSOR && !nstate_tensor_applies(a)) return DSLA_ERR_UNSUPPORTED;
     if (st->n_states != a->n_states || st->H != a->H || st->d_k != a->d_k || st->d_v != a->d_v) return DSLA_ERR_INVALID_ARG;
     if (!a->slots && a->N > st->num_slots) return DSLA_ERR_INVALID_ARG;
     if (!(a->scale == a->scale) || !on_store_device(st)) return DSLA_ERR_INVALID_ARG;
@@ -298,6 +356,40 @@ dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* s
     if (a->T_total > 0) {
         if (!a->q || !a->k || !a->v || !a->o || !a->gates) return DSLA_ERR_INVALID_ARG;
         if (!aligned(a->q, 16) || !aligned(a->k, 16) || !aligned(a->v, 16) || !aligned(a->o, 16)) return DSLA_ERR_INVALID_ARG;
+    }
+    if (a->impl != DSLA_IMPL_SIMT && nstate_tensor_applies(a) && a->T_total > 0) {
+        const dsla_prefill_args b = nstate_as_prefill_args(a);
+        const size_t need_tc = prefill_tc_workspace_bytes(&b, false), need = need_tc + nstate_o_scratch_bytes(a);
+        if (need > 0 && (!a->workspace || a->workspace_bytes < need || !aligned(a->workspace, 256))) return DSLA_ERR_INVALID_ARG;
+        if (!aligned(a->gates, 4)) return DSLA_ERR_INVALID_ARG;
+        void* o_scratch = static_cast<char*>(a->workspace) + need_tc;
+        const size_t n8 = (size_t)a->T_total * a->H * a->d_v / 8;
+        cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+        PrefillParams p{};
+        p.q = a->q; p.k = a->k; p.v = a->v; p.o = a->o;
+        p.gamma = nullptr; p.cu_seqlens = a->cu_seqlens; p.slots = a->slots;
+        p.state = st->data; p.status = st->status;
+        p.N = a->N; p.T = a->T; p.H = a->H; p.num_slots = st->num_slots;
+        p.max_chunks = (a->max_seqlen + 63) / 64;
+        p.scale = a->scale; p.use_initial_state = a->use_initial_state ? 1 : 0;
+        p.weights = a->weights; p.n_total = a->n_states;
+        const size_t gs = (size_t)a->T_total * a->H;
+        for (int first = 0; first < a->n_states; first += 2) {      // one pass of the dual-state kernel per pair of states
+            p.g_hist = a->gates + (size_t)first * gs;
+            p.g_rec = a->gates + (size_t)(first + 1) * gs;
+            p.state_first = first;
+            p.o = first == 0 ? a->o : o_scratch;
+            const dsla_status rc = launch_prefill_tc(p, &b, false, s);
+            if (rc != DSLA_OK) return rc;
+            if (first > 0) {
+                const size_t blocks = (n8 + 255) / 256;
+                add_bf16_kernel<<<dim3((unsigned)(blocks < 148 * 8 ? blocks : 148 * 8)), dim3(256), 0, s>>>(
+                    static_cast<uint4*>(a->o), static_cast<const uint4*>(o_scratch), n8);
+                count_launch();
+                if (cudaGetLastError() != cudaSuccess) return DSLA_ERR_CUDA;
+            }
+        }
+        return DSLA_OK;
     }
     RecurrentParams r{};
     r.q = a->q; r.k = a->k; r.v = a->v; r.o = a->o;

@@ -23,12 +23,16 @@ struct PrefillParams {
     const float *g_hist, *g_rec, *gamma;
     const int32_t* cu_seqlens;  // may be null (dense)
     const int32_t* slots;       // may be null
-    float* state;               // [num_slots][2][H][D][D]
+    float* state;               // [num_slots][n_total][H][D][D]; this call works on states state_first, state_first + 1
     int* status;
     int N, T, H, num_slots;
     int max_chunks;             // ceil(max_seqlen / C)
     float scale;
     int use_initial_state;
+    // n-state form run two states at a time (tensor-core kernel only; the dual-state path leaves the defaults)
+    const float* weights;       // [H, n_total] blend weights, or nullptr: (gamma, 1 - gamma)
+    int n_total;                // states per slot (2 for the dual-state layer)
+    int state_first;            // index of the first of the two states of this call
 };
 
 struct DecodeParams {

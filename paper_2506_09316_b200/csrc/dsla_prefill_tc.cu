@@ -86,7 +86,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const SeqInfo sq = seq_info(p, n, g, tp.nseg, tp.cps, tp.skew8);
     if (sq.slot < 0 || sq.slot >= p.num_slots) return;
     if (tid == 0 && g == 0 && sq.nchunks > seg_begin(tp.nseg, tp.nseg, tp.cps, tp.skew8)) atomicExch(p.status, (int)DSLA_ERR_INVALID_ARG);
-    float* slot1 = p.state + (((size_t)sq.slot * 2) * p.H + h) * (size_t)(D * D);
+    float* slot1 = p.state + (((size_t)sq.slot * p.n_total + p.state_first) * p.H + h) * (size_t)(D * D);
     const size_t state_stride = (size_t)p.H * D * D;
     // where the initial state is read: the slot, or the snapshot taken before this grid (split sequences)
     const float* init1 = tp.init ? tp.init + (size_t)(n * p.H + h) * 2 * (size_t)(D * D) : slot1;
@@ -337,8 +337,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // triangle of 32..63; the full block (rows 32..63, columns 0..31) factors through token 31,
         // 2^(L_j - L_31) 2^(L_31 - L_s) with both factors <= 1, and is split between the two warps.
         const int gw = warp - GATE_W0;
-        const float gam = p.gamma[h];
-        const float W1 = gam * p.scale, W2 = (1.f - gam) * p.scale;
+        const float W1 = (p.weights ? p.weights[(size_t)h * p.n_total + p.state_first] : p.gamma[h]) * p.scale;
+        const float W2 = (p.weights ? p.weights[(size_t)h * p.n_total + p.state_first + 1] : 1.f - p.gamma[h]) * p.scale;
         auto fetch = [&](int c, float2& lo, float2& hi2) {
             const int j = c * C + lane;
             const bool in = c < nc;

@@ -172,8 +172,11 @@ def test_tensor_kernels_refuse_per_key_channel_gates():
 
 
 @pytest.mark.parametrize("n", [1, 2, 4, 8])
-@pytest.mark.parametrize("dtype,d,vec", [(F32, 64, False), (BF, 128, False), (BF, 128, True), (F32, 64, True)])
-def test_nstate_prefill(n, dtype, d, vec):
+@pytest.mark.parametrize("dtype,d,vec,impl", [(F32, 64, False, "auto"), (BF, 128, False, "auto"), (BF, 128, False, "simt"), (BF, 128, True, "auto"),
+                                               (F32, 64, True, "auto")])
+def test_nstate_prefill(n, dtype, d, vec, impl):
+    """bf16, d = 128, scalar gates, even n: AUTO runs the chunkwise tensor-core kernel once per pair of states; everything
+    else (and impl="simt") the token-by-token kernel."""
     import paper_2506_09316_b200 as dsla
     rng = np.random.default_rng(3700 + n + d)
     lens = [33, 0, 150, 1]
@@ -189,8 +192,9 @@ def test_nstate_prefill(n, dtype, d, vec):
     dv = inp.to("cuda")
     o = dsla.dsla_nstate_prefill(dv.q, dv.k, dv.v, torch.from_numpy(gates).cuda(), torch.from_numpy(w).cuda(), st,
                                  cu_seqlens=dv.cu_seqlens, slots=torch.from_numpy(slots).cuda(), scale=0.8,
-                                 use_initial_state=True)
+                                 use_initial_state=True, impl=impl, max_seqlen=max(lens))
     torch.cuda.synchronize()
+    assert dsla.dsla_state_last_error(st) == dsla.DSLA_OK
     f = inp.as_f64()
     ref_state = st0.astype(np.float64)
     o_ref, S_ref = orc.prefill_n(f["q"], f["k"], f["v"], gates, w, f["cu_seqlens"], scale=0.8, state=ref_state, slots=slots)
@@ -198,6 +202,40 @@ def test_nstate_prefill(n, dtype, d, vec):
     tol = TOL[dtype] * (1.5 if (dtype == BF and n == 8) else 1.0)
     assert rel_err(_f64(o), o_ref) <= tol
     assert rel_err(_f64(st.tensor), S_ref) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("n,use_init", [(2, False), (4, True), (8, False)])
+def test_nstate_prefill_tensor_path_with_split_sequences(n, use_init):
+    """Few (sequence, head) pairs and long sequences: every pair of states runs the summary pass, the fold and (on a
+    resume) the snapshot of its own two states; pairs after the first add to the output."""
+    import paper_2506_09316_b200 as dsla
+    rng = np.random.default_rng(3750 + n)
+    lens = [1500, 64, 777]
+    H, d = 2, 128
+    inp = gen.make_packed(3751 + n, lens, H, d, BF)
+    T = inp.T_total
+    gates = (1.0 / (1.0 + np.exp(-rng.normal(3.0, 1.5, size=(n, T, H))))).astype(np.float32)
+    gates[:, 100, :] = 0.0
+    gates[:, 900:910, 0] = 1.0
+    w = rng.normal(size=(H, n)).astype(np.float32)
+    st0 = (rng.normal(size=(3, n, H, d, d)) * 0.3).astype(np.float32)
+    st = dsla.dsla_state_alloc_n(3, n, H, d, d)
+    st.tensor.copy_(torch.from_numpy(st0))
+    dv = inp.to("cuda")
+    o = dsla.dsla_nstate_prefill(dv.q, dv.k, dv.v, torch.from_numpy(gates).cuda(), torch.from_numpy(w).cuda(), st,
+                                 cu_seqlens=dv.cu_seqlens, max_seqlen=max(lens), use_initial_state=use_init, impl="tensor")
+    torch.cuda.synchronize()
+    assert dsla.dsla_state_last_error(st) == dsla.DSLA_OK
+    f = inp.as_f64()
+    ref_state = st0.astype(np.float64) if use_init else np.zeros_like(st0, dtype=np.float64)
+    o_ref, S_ref = orc.prefill_n(f["q"], f["k"], f["v"], gates, w, f["cu_seqlens"], state=ref_state)
+    assert rel_err(_f64(o), o_ref) <= TOL[BF] * (1.5 if n == 8 else 1.0)
+    assert rel_err(_f64(st.tensor), S_ref) <= TOL[BF]
+    # the tensor path is refused where it does not apply
+    with pytest.raises(dsla.DslaError) as e:
+        dsla.dsla_nstate_prefill(dv.q, dv.k, dv.v, torch.ones(1, T, H, device="cuda"), torch.ones(H, 1, device="cuda"),
+                                 dsla.dsla_state_alloc_n(3, 1, H, d, d), cu_seqlens=dv.cu_seqlens, max_seqlen=max(lens), impl="tensor")
+    assert e.value.status == dsla.DSLA_ERR_UNSUPPORTED
 
 
 def test_nstate_entry_points_check_the_store():
