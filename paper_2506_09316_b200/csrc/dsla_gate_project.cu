@@ -4,8 +4,8 @@
 // written straight in the [T, H] fp32 layout the prefill and decode kernels read, so no pre-activation tensor
 // crosses HBM.  A tcgen05 GEMM: CTA = 128 tokens, M = 128 (tokens on the TMEM lanes), N = 2 H, K = D_model in
 // steps of 64; TMA lands the x and W tiles (128-byte swizzle) in a four-stage ring; the epilogue reads the fp32
-// accumulator from TMEM (one token per thread), adds the bias, applies the logistic and stores 128 contiguous bytes
-// per thread and gate tensor.  Bound by reading x once from HBM (T * D_model * 2 bytes).
+// accumulator from TMEM (one token per thread), adds the bias, applies the logistic and stores 16 bytes at a time (the
+// H outputs of a token and gate tensor are contiguous).  Bound by reading x once from HBM (T * D_model * 2 bytes).
 //
 // Few tokens mean few CTAs (32 at T = 4096), and one CTA streams its rows at a fraction of what the SM could
 // take: then K is split over the 2 or 4 CTAs of a thread-block cluster.  Each CTA accumulates its share of the
