@@ -7,26 +7,31 @@
 // of the Sec. 4.1 recurrence.  The chunks are walked from the END of the segment backwards while a
 // running product R^i of all later gates is carried, so every token's weight prod_{t > s} g^i_t (to the
 // end of the segment) is a plain product: no logarithms, no rescaling of the accumulator, and a zero
-// gate is exact.  A pure streaming pipeline, four chunks deep: warps 10, 11 derive the weights (one
-// state each), warps 0..7 scale K into the two weighted copies, warp 8 drives TMA, warp 9 issues the
-// MMAs  [S1^T | S2^T] += V^T [K~1 | K~2]  (M = 128, N = 256, K = 64 tokens).
+// gate is exact.  A pure streaming pipeline: warps 10, 11 derive the weights (one state each), warps
+// 0..3 build the weighted, transposed V~i^T of both states in TMEM straight from the V tile (ldmatrix
+// with .trans hands a thread two consecutive tokens of one d_v column, which is the element pair a
+// 16x128b TMEM store takes: no shuffles and no scaled copy in shared memory), warp 8 drives TMA,
+// warp 9 issues the MMAs  S^i^T += V~i^T K  (M = 128, N = 128, K = 64 tokens; A in TMEM, B = the raw
+// K tile), warps 4..7 only help with the final store.
 #include "dsla_prefill_tc.cuh"
 
 namespace dsla {
 
 namespace {
 
-constexpr int SUM_STAGES = 4, SUM_STAGE_BYTES = 3 * 16384, SUM_OFF_V = 32768;   // stage = [K/K~1][K~2][V]
-constexpr int SUM_NTHREADS = 384, SUM_NCOMPUTE = 256;
+constexpr int SUM_STAGES = 6, SUM_STAGE_BYTES = 2 * 16384, SUM_OFF_V = 16384;   // stage = [K][V]
+constexpr int SUM_WSTAGES = 4;           // ring of per-chunk weights
+constexpr int SUM_NTHREADS = 384;
 constexpr int SUM_GATE_AHEAD = 6;        // chunks between the L2 prefetch and the load of a chunk's gates
 constexpr int SUM_PREFETCH = 8;          // chunks between the L2 prefetch and the load of a tile
 constexpr int SUM_SMEM_DYN = SUM_STAGES * SUM_STAGE_BYTES + 1024;
+constexpr uint32_t SUM_COL_VT = 256;     // V~^T, bf16: [chunk parity][state] x 32 columns
 
 struct alignas(16) SumShared {
-    uint64_t full[SUM_STAGES], empty[SUM_STAGES], w_ready[SUM_STAGES], w_free[SUM_STAGES], k_ready[SUM_STAGES], u_full;
+    uint64_t full[SUM_STAGES], empty[SUM_STAGES], w_ready[SUM_WSTAGES], w_free[SUM_WSTAGES], vt_ready[2], vt_free[2], u_full;
     uint32_t tmem_base;
     int abort_flag;
-    uint32_t wts[SUM_STAGES][2][C];     // per-token weights, bf16 in both halves
+    __nv_bfloat16 wts[SUM_WSTAGES][2][C];     // per-token weights
 };
 
 __global__ void __launch_bounds__(SUM_NTHREADS, 1)
@@ -50,22 +55,21 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     float* out = tp.ws + ((size_t)(n * p.H + h) * tp.nseg + g) * (SUMMARY_STRIDE / 4);
 
     if (tid == 0) {
-        for (int s = 0; s < SUM_STAGES; ++s) {
-            mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1);
-            mbar_init(&sh.w_ready[s], 2); mbar_init(&sh.w_free[s], 8); mbar_init(&sh.k_ready[s], 8);
-        }
+        for (int s = 0; s < SUM_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 5); }   // four V~ warps + the MMAs on K
+        for (int s = 0; s < SUM_WSTAGES; ++s) { mbar_init(&sh.w_ready[s], 2); mbar_init(&sh.w_free[s], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&sh.vt_ready[b], 4); mbar_init(&sh.vt_free[b], 1); }
         mbar_init(&sh.u_full, 1);
         sh.abort_flag = 0;
         fence_barrier_init();
     }
-    if (warp == 9) { tmem_alloc(&sh.tmem_base, 256); tmem_relinquish(); }
+    if (warp == 9) { tmem_alloc(&sh.tmem_base, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = sh.tmem_base;
     volatile int* abortp = &sh.abort_flag;
 
-    // iteration it = 0 .. nc-1 handles chunk nc-1-it; stage s = it % 4, use u = it / 4 of that stage
+    // iteration it = 0 .. nc-1 handles chunk nc-1-it; tile stage it % 6, weight stage it % 4, V~ buffer it % 2
     if (warp == 8) {
         if (lane == 0) {
             prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
@@ -75,9 +79,9 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
                 uint8_t* st = tiles + s * SUM_STAGE_BYTES;
                 const int t = t0 + (nc - 1 - it) * C;
                 mbar_arrive_expect_tx(&sh.full[s], 4 * 8192);
-                tma_load_4d(st, &map_k, &sh.full[s], 0, t, 0, h);
                 tma_load_4d(st + SUM_OFF_V, &map_v, &sh.full[s], 0, t, 0, h);
-                if (it + SUM_PREFETCH < nc) {   // pull a tile well ahead into L2: the four stages alone do not cover the HBM latency
+                tma_load_4d(st, &map_k, &sh.full[s], 0, t, 0, h);
+                if (it + SUM_PREFETCH < nc) {   // pull a tile well ahead into L2: the stages alone do not cover the HBM latency
                     const int tp2 = t - SUM_PREFETCH * C;
                     tma_prefetch_4d(&map_k, 0, tp2, 0, h);
                     tma_prefetch_4d(&map_v, 0, tp2, 0, h);
@@ -87,16 +91,20 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     } else if (warp == 9) {
         if (lane == 0) {
             const uint32_t sa = smem_u32(tiles);
-            constexpr uint32_t ID_U = idesc_bf16(128, 256, 1, 1);
+            constexpr uint32_t ID_U = idesc_bf16(128, 128, 0, 1);       // A in TMEM, B = K as an MN-major N operand
             for (int it = 0; it < nc; ++it) {
-                const int s = it % SUM_STAGES, u = it / SUM_STAGES;
-                mbar_wait(&sh.k_ready[s], u & 1, abortp, p.status);
+                const int s = it % SUM_STAGES, u = it / SUM_STAGES, b = it & 1;
+                mbar_wait(&sh.full[s], u & 1, abortp, p.status);
+                mbar_wait(&sh.vt_ready[b], (it >> 1) & 1, abortp, p.status);
                 tc_fence_after();
-                const uint32_t st = sa + s * SUM_STAGE_BYTES;
-                const uint64_t dv = smem_desc_sw128(st + SUM_OFF_V, 8192, 1024), dkk = smem_desc_sw128(st, 8192, 1024);
+                const uint64_t dkk = smem_desc_sw128(sa + s * SUM_STAGE_BYTES, 8192, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) mma_ss(tb, dv + (uint64_t)(kk * 128), dkk + (uint64_t)(kk * 128), ID_U, (it | kk) > 0);
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ts(tb + 128 * i, tb + SUM_COL_VT + 64 * b + 32 * i + 8 * kk, dkk + (uint64_t)(kk * 128), ID_U, (it | kk) > 0);
                 tc_commit(&sh.empty[s]);
+                tc_commit(&sh.vt_free[b]);
                 if (it == nc - 1) tc_commit(&sh.u_full);
             }
         }
@@ -109,7 +117,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
         float n0 = load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane, p.H, h, true);     // raw; clamped where it is used
         float n1 = load_gate(gsrc, t0 + (nc - 1) * C + 2 * lane + 1, p.H, h, true);
         for (int it = 0; it < nc; ++it) {
-            const int s = it % SUM_STAGES, u = it / SUM_STAGES;
+            const int s = it % SUM_WSTAGES, u = it / SUM_WSTAGES;
             const float g0 = fmaxf(n0, 0.f), g1 = fmaxf(n1, 0.f);
             if (it + 1 < nc) {
                 const int t = t0 + (nc - 2 - it) * C + 2 * lane;
@@ -129,34 +137,61 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
             if (lane == 31) ex = 1.f;
             ex *= R;
             if (u >= 1) mbar_wait(&sh.w_free[s], (u - 1) & 1, abortp, p.status);
-            *reinterpret_cast<uint2*>(&sh.wts[s][i][2 * lane]) = make_uint2(dup_bf16(g1 * ex), dup_bf16(ex));
+            *reinterpret_cast<__nv_bfloat162*>(&sh.wts[s][i][2 * lane]) = __floats2bfloat162_rn(g1 * ex, ex);
             R *= tot;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.w_ready[s]);
         }
         if (lane == 0) out[2 * D * D + i] = R;         // A_g: product of every gate of the segment
     } else {
-        // ---- K~1 (in place) and K~2: four 16-byte pieces per thread and chunk
         const int q = warp & 3, hi = warp >> 2;
         const uint32_t lane_addr = tb + ((uint32_t)(32 * q) << 16);
-        for (int it = 0; it < nc; ++it) {
-            const int s = it % SUM_STAGES, u = it / SUM_STAGES;
-            uint8_t* st = tiles + s * SUM_STAGE_BYTES;
-            mbar_wait(&sh.w_ready[s], u & 1, abortp, p.status);
-            mbar_wait(&sh.full[s], u & 1, abortp, p.status);
+        if (warp < 4) {
+            // ---- V~i^T[v][s] = w^i_s V[s][v] for both states into TMEM (d_v on the lanes, two tokens per 32-bit column).
+            // One round = 16 tokens x 16 d_v lanes: matrices (tokens 0..7 | 8..15) x (d_v 0..7 | 8..15); a 16x128b TMEM store
+            // takes the ldmatrix.trans distribution as it is (lane = t / 4, column = t % 4).
+            const int mk = lane >> 3, mr = lane & 7;                 // this thread addresses row mr of matrix mk
+            for (int it = 0; it < nc; ++it) {
+                const int s = it % SUM_STAGES, u = it / SUM_STAGES, ws = it % SUM_WSTAGES, b = it & 1;
+                mbar_wait(&sh.w_ready[ws], (it / SUM_WSTAGES) & 1, abortp, p.status);
+                mbar_wait(&sh.full[s], u & 1, abortp, p.status);
+                if (it >= 2) mbar_wait(&sh.vt_free[b], ((it >> 1) - 1) & 1, abortp, p.status);     // the MMAs of chunk it - 2 have read this buffer
+                tc_fence_after();
+                const uint32_t vtile = smem_u32(tiles + s * SUM_STAGE_BYTES + SUM_OFF_V);
+                const uint8_t* wp0 = reinterpret_cast<const uint8_t*>(sh.wts[ws][0]) + 4 * (lane & 3);
+                const uint8_t* wp1 = reinterpret_cast<const uint8_t*>(sh.wts[ws][1]) + 4 * (lane & 3);
+#pragma unroll 1
+                for (int hh = 0; hh < 2; ++hh) {       // the two 16-lane halves of this warp's TMEM quadrant
+                    const int d = 32 * q + 16 * hh + 8 * (mk & 1);            // first d_v column of the matrix this thread addresses
+                    // row of the V tile: token * 128 bytes, 16-byte piece (d / 8 mod 8) ^ (token mod 8); token mod 8 = mr in every round
+                    const uint32_t row0 = vtile + (uint32_t)(d >> 6) * 8192u + (uint32_t)((8 * (mk >> 1) + mr) * 128) +
+                                          (((uint32_t)((d & 63) >> 3) ^ (uint32_t)mr) << 4);
+                    const uint32_t vt = tb + ((uint32_t)(32 * q + 16 * hh) << 16) + SUM_COL_VT + 64 * b;
+                    uint32_t r[16];
 #pragma unroll
-            for (int m = 0; m < 4; ++m) {
-                const int idx = tid + SUM_NCOMPUTE * m;
-                const int row = (idx >> 3) & 63;
-                uint4* kp = reinterpret_cast<uint4*>(st) + idx;
-                const uint4 xk = *kp;
-                const uint32_t w0 = sh.wts[s][0][row], w1 = sh.wts[s][1][row];
-                *kp = scale8(xk, w0);
-                *(kp + 1024) = scale8(xk, w1);
+                    for (int t16 = 0; t16 < 4; ++t16)      // all loads of the half first: their latencies overlap
+                        ldmatrix_x4_trans(row0 + (uint32_t)(t16 * 16 * 128), r[4 * t16], r[4 * t16 + 1], r[4 * t16 + 2], r[4 * t16 + 3]);
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const uint8_t* wp = i == 0 ? wp0 : wp1;
+#pragma unroll
+                        for (int t16 = 0; t16 < 4; ++t16) {
+                            const __nv_bfloat162 ww0 = *reinterpret_cast<const __nv_bfloat162*>(wp + 32 * t16);
+                            const __nv_bfloat162 ww1 = *reinterpret_cast<const __nv_bfloat162*>(wp + 32 * t16 + 16);
+                            const __nv_bfloat162 y0 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16]), ww0);
+                            const __nv_bfloat162 y1 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16 + 1]), ww0);
+                            const __nv_bfloat162 y2 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16 + 2]), ww1);
+                            const __nv_bfloat162 y3 = __hmul2(*reinterpret_cast<const __nv_bfloat162*>(&r[4 * t16 + 3]), ww1);
+                            tmem_st_16x128b(vt + 32 * i + 8 * t16, *reinterpret_cast<const uint32_t*>(&y0), *reinterpret_cast<const uint32_t*>(&y1));
+                            tmem_st_16x128b(vt + 32 * i + 8 * t16 + 4, *reinterpret_cast<const uint32_t*>(&y2), *reinterpret_cast<const uint32_t*>(&y3));
+                        }
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(&sh.vt_ready[b]); mbar_arrive(&sh.empty[s]); mbar_arrive(&sh.w_free[ws]); }
             }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(&sh.k_ready[s]); mbar_arrive(&sh.w_free[s]); }
         }
         mbar_wait(&sh.u_full, 0, abortp, p.status);
         tc_fence_after();
@@ -164,7 +199,7 @@ prefill_tc_summary_kernel(const __grid_constant__ CUtensorMap map_k, const __gri
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tb, 256);
+    if (warp == 9) tmem_dealloc(tb, 512);
 }
 
 // Ragged batches: blocks are handed to the SMs in index order, so sequences are visited longest first (a long
