@@ -241,12 +241,16 @@ def extra_prefill_section(dsla, name, kernel, steps, dev, rank, peaks, dense=Non
     """A further prefill workload reported beside the headline one: median and best of the per-step event times."""
     spec = workload_spec(name, dense)
     r = time_prefill(dsla, spec, kernel, steps, 3, dev, rank, peaks)
-    stream = torch.cuda.current_stream()
+    time.sleep(0.2)          # let the power state of the section before settle; the clocks of this section are sampled below
+    sampler = ClockSampler(visible_nvml_index(dev.index or 0))
+    sampler.start()
     for i in range(steps):
         r["step"](i, r["evs"][i])
     torch.cuda.synchronize()
+    clocks = sampler.stop()
     ms = [e[0].elapsed_time(e[1]) for e in r["evs"]]
     out = {"workload": f"{dense or name}: N={r['N']} H={spec['H']} d={spec['d']} T_total={r['T_total']}", "kernel": kernel, "steps": steps,
+           "clocks": clocks,
            "median": prefill_numbers(r["T_total"], spec["H"], spec["d"], float(np.median(ms)), peaks),
            "best": prefill_numbers(r["T_total"], spec["H"], spec["d"], float(np.min(ms)), peaks)}
     del r
@@ -330,10 +334,10 @@ def bench_ours(args):
         other = "pair" if args.kernel != "pair" else "tensor"
         if not args.dense:
             more[f"{args.workload}_{other}"] = extra_prefill_section(dsla, args.workload, other, 10, dev, rank, peaks)
-        for name in ("cfg3", "cfg5"):
+        more["dense_4x37x16384"] = extra_prefill_section(dsla, "cfg2", args.kernel, 10, dev, rank, peaks, dense="4,37,16384")
+        for name in ("cfg3", "cfg5"):      # the heaviest section last
             if name != args.workload or args.dense:
                 more[name] = extra_prefill_section(dsla, name, args.kernel, 5, dev, rank, peaks)
-        more["dense_4x37x16384"] = extra_prefill_section(dsla, "cfg2", args.kernel, 5, dev, rank, peaks, dense="4,37,16384")
 
     decode = None
     if not args.no_decode:
