@@ -74,6 +74,7 @@ __global__ void __launch_bounds__(256) prefill_recurrent_kernel(const RecurrentP
             if (!VG && c < NSG) sg[c][j][0] = fmaxf(p.g[c][(size_t)(t_begin + c0 + j) * p.H + h], 0.f);
         }
         __syncthreads();
+#pragma unroll 4      // four tokens in flight: their shuffle reductions overlap (8 spills with vector gates)
         for (int j = 0; j < nt; ++j) {
             const float4 vv = *reinterpret_cast<const float4*>(&sv[j][4 * warp]);
             float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
