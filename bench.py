@@ -570,16 +570,17 @@ def bench_extensions(dsla, peaks, dev, rank):
     t = timed(lambda: dsla.dsla_prefill(pin.q, pin.k, pin.v, gc1, gc2, pin.gamma, st, o=oo, max_seqlen=T), steps=5)
     out["prefill_per_key_channel_gates"] = {"workload": f"N=1 H={H} d={d} T={T} bf16", "ms": t * 1e3, "tokens_per_s": T / t,
                                             "kernel": "token-by-token CUDA-core recurrence"}
-    for n in (2, 4):
+    for n in (1, 2, 4, 8):
         stn = dsla.dsla_state_alloc_n(1, n, H, d, d, device=dev)
         gates = torch.sigmoid(torch.randn((n, T, H), generator=g, device=dev) * 0.5 + 3.0)
         w = torch.rand((H, n), generator=g, device=dev)
         ws = torch.empty(max(1, dsla.dsla_nstate_prefill_workspace_bytes(pin.q, pin.k, pin.v, gates, w, max_seqlen=T)), dtype=torch.uint8, device=dev)
         t = timed(lambda: dsla.dsla_nstate_prefill(pin.q, pin.k, pin.v, gates, w, stn, o=oo, max_seqlen=T, workspace=ws), steps=10)
         t2 = timed(lambda: dsla.dsla_nstate_prefill(pin.q, pin.k, pin.v, gates, w, stn, o=oo, max_seqlen=T, impl="simt"), steps=3)
-        flops = T * H * (2 * 64 * 2 * d + n * 4 * d * d) * (n // 2) / max(n // 2, 1) if n < 2 else T * H * (n // 2) * FLOP_PER_TOKEN_HEAD(d, 64)
+        passes = max(1, n // 2)
+        flops = T * H * passes * FLOP_PER_TOKEN_HEAD(d, 64)      # what the kernel executes: every pass is a full dual-state pass
         out[f"prefill_{n}_states"] = {"workload": f"N=1 H={H} d={d} T={T} bf16, scalar gates", "ms": t * 1e3, "tokens_per_s": T / t,
-                                      "kernel": f"chunkwise tensor-core kernel, {n // 2} pass(es) of two states",
+                                      "kernel": f"chunkwise tensor-core kernel, {passes} pass(es) of two states",
                                       "executed_tflops": flops / t / 1e12, "token_by_token_kernel_ms": t2 * 1e3}
         del stn, ws
     return out

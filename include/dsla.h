@@ -259,7 +259,8 @@ typedef struct {
  *  - SIMT: the recurrence itself on CUDA cores, token by token (fp32 arithmetic, no workspace), for every supported
  *    n, dtype, d and gate layout.  With more than four states (more than two when the gates are per key channel and
  *    d = 128) the states are processed in groups, each group adding its share to o.
- *  - TENSOR (what AUTO picks when it applies): bf16, d = 128, scalar gates, n in {2, 4, 8}: the chunkwise tensor-core
+ *  - TENSOR (what AUTO picks when it applies): bf16, d = 128, scalar gates (n = 1 runs as a pair whose second state
+ *    has weight 0 and is never stored): the chunkwise tensor-core
  *    kernel of dsla_prefill run once per pair of states (2i, 2i + 1) with the weights (w_2i, w_2i+1); pairs after the
  *    first write their share to a scratch tensor in the workspace that is then added to o, so o is rounded to bf16 once
  *    per pair.  Needs the workspace below.

@@ -421,9 +421,9 @@ def dsla_nstate_prefill_workspace_bytes(q, k, v, gates, weights, *, cu_seqlens=N
 
 def dsla_nstate_prefill(q, k, v, gates, weights, st: DslaState, *, o=None, cu_seqlens=None, slots=None, max_seqlen=None,
                         scale=1.0, use_initial_state=False, impl="auto", workspace=None, stream=None):
-    """n-state prefill: gates [n, T_total, H] (or [n, T_total, H, d] per key channel), weights [H, n].  bf16, d = 128,
-    scalar gates and an even n run on the chunkwise tensor-core kernel, one pass per pair of states (``impl="simt"``
-    forces the token-by-token CUDA-core kernel, which serves everything else)."""
+    """n-state prefill: gates [n, T_total, H] (or [n, T_total, H, d] per key channel), weights [H, n].  bf16, d = 128
+    with scalar gates runs on the chunkwise tensor-core kernel, one pass per pair of states (``impl="simt"`` forces the
+    token-by-token CUDA-core kernel, which serves everything else)."""
     if o is None:
         o = torch.empty_like(v)
     a = _nstate_prefill_args(q, k, v, o, gates, weights, cu_seqlens, slots, max_seqlen, scale, use_initial_state, impl)

@@ -221,7 +221,7 @@ static dsla_status prefill_device(const dsla_prefill_args* a, dsla_state* st, cu
     const int chunk = a->chunk == 0 ? 64 : a->chunk;
     p.max_chunks = (a->max_seqlen + chunk - 1) / chunk;
     p.scale = a->scale; p.use_initial_state = a->use_initial_state ? 1 : 0;
-    p.weights = nullptr; p.n_total = 2; p.state_first = 0;
+    p.weights = nullptr; p.n_total = 2; p.state_first = 0; p.single = 0;
     if (a->gate_layout == DSLA_GATE_PER_KEY_CHANNEL) {
         // the dual state as two states whose weights the kernel derives from gamma: (gamma, 1 - gamma)
         RecurrentParams r{};
@@ -327,9 +327,9 @@ static dsla_status check_nstate_prefill_sizes(const dsla_nstate_prefill_args* a)
     return DSLA_OK;
 }
 
-// pairs of states through the chunkwise tensor-core kernel: bf16, d = 128, scalar gates, an even number of states
+// pairs of states (or the single state) through the chunkwise tensor-core kernel: bf16, d = 128, scalar gates
 static bool nstate_tensor_applies(const dsla_nstate_prefill_args* a) {
-    return a->dtype == DSLA_BF16 && a->d_k == 128 && a->gate_layout == DSLA_GATE_SCALAR && a->n_states % 2 == 0 && prefill_tc_available();
+    return a->dtype == DSLA_BF16 && a->d_k == 128 && a->gate_layout == DSLA_GATE_SCALAR && prefill_tc_available();
 }
 
 // pairs after the first write their share of o to a scratch tensor that is then added to o
@@ -376,7 +376,8 @@ dsla_status dsla_nstate_prefill(const dsla_nstate_prefill_args* a, dsla_state* s
         const size_t gs = (size_t)a->T_total * a->H;
         for (int first = 0; first < a->n_states; first += 2) {      // one pass of the dual-state kernel per pair of states
             p.g_hist = a->gates + (size_t)first * gs;
-            p.g_rec = a->gates + (size_t)(first + 1) * gs;
+            p.single = a->n_states == 1;
+            p.g_rec = a->gates + (size_t)(p.single ? first : first + 1) * gs;
             p.state_first = first;
             p.o = first == 0 ? a->o : o_scratch;
             const dsla_status rc = launch_prefill_tc(p, &b, false, s);

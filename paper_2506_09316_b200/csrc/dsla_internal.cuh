@@ -33,6 +33,8 @@ struct PrefillParams {
     const float* weights;       // [H, n_total] blend weights, or nullptr: (gamma, 1 - gamma)
     int n_total;                // states per slot (2 for the dual-state layer)
     int state_first;            // index of the first of the two states of this call
+    int single;                 // only state_first exists (n = 1): the second state of the kernel runs with weight 0 on the first
+                                // state's gates, starts from zero and is never loaded from or stored to the slot
 };
 
 struct DecodeParams {

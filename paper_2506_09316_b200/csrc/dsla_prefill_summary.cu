@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(256) state_snapshot_kernel(const PrefillParams
     const int unit = blockIdx.x >> 1, i = blockIdx.x & 1;
     const int n = unit / p.H, h = unit % p.H;
     const int slot = p.slots ? p.slots[n] : n;
-    if (slot < 0 || slot >= p.num_slots) return;
+    if (slot < 0 || slot >= p.num_slots || (p.single && i == 1)) return;
     const float4* src = reinterpret_cast<const float4*>(p.state + (((size_t)slot * p.n_total + p.state_first + i) * p.H + h) * (size_t)(D * D));
     float4* dst = reinterpret_cast<float4*>(snap + ((size_t)unit * 2 + i) * (size_t)(D * D));
     for (int k = threadIdx.x; k < D * D / 4; k += 256) dst[k] = src[k];

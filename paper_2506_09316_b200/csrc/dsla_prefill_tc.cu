@@ -93,7 +93,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const size_t init_stride = tp.init ? (size_t)(D * D) : state_stride;
     if (sq.len <= 0) {  // empty sequence: a fresh start leaves zero states, a resume leaves the slot alone
         if (g == 0 && !p.use_initial_state)
-            for (int i = tid; i < 2 * D * D; i += NTHREADS) slot1[(size_t)(i / (D * D)) * state_stride + i % (D * D)] = 0.f;
+            for (int i = tid; i < (p.single ? 1 : 2) * D * D; i += NTHREADS) slot1[(size_t)(i / (D * D)) * state_stride + i % (D * D)] = 0.f;
         return;
     }
     if (sq.c_begin >= sq.c_end) return;
@@ -255,7 +255,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) a0 *= __shfl_xor_sync(0xffffffffu, a0, off);      // decay of chunk 0
             if (g > 0 && tp.ws) asm volatile("griddepcontrol.wait;" ::: "memory");
-            init_state_pass(init1 + (size_t)half * init_stride, p.use_initial_state,
+            init_state_pass(init1 + (size_t)half * init_stride, p.use_initial_state && !(p.single && half == 1),
                             tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, half, 32 * q + lane, a0,
                             lane_addr + COL_S + 128 * half, lane_addr + COL_SB + 64 * half, 2, 4);
             tc_wait_st();
@@ -338,7 +338,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // 2^(L_j - L_31) 2^(L_31 - L_s) with both factors <= 1, and is split between the two warps.
         const int gw = warp - GATE_W0;
         const float W1 = (p.weights ? p.weights[(size_t)h * p.n_total + p.state_first] : p.gamma[h]) * p.scale;
-        const float W2 = (p.weights ? p.weights[(size_t)h * p.n_total + p.state_first + 1] : 1.f - p.gamma[h]) * p.scale;
+        const float W2 = p.single ? 0.f : (p.weights ? p.weights[(size_t)h * p.n_total + p.state_first + 1] : 1.f - p.gamma[h]) * p.scale;
         auto fetch = [&](int c, float2& lo, float2& hi2) {
             const int j = c * C + lane;
             const bool in = c < nc;
@@ -454,7 +454,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // With programmatic dependent launch this grid may start while the summary grid is still running;
                 // everything up to here (and all of chunk 0's operand work in the other warps) is independent of it.
                 if (g > 0 && tp.ws) asm volatile("griddepcontrol.wait;" ::: "memory");
-                init_state_pass(init1 + (size_t)hi * init_stride, p.use_initial_state,
+                init_state_pass(init1 + (size_t)hi * init_stride, p.use_initial_state && !(p.single && hi == 1),
                                 tp.ws ? tp.ws + ((size_t)(n * p.H + h) * tp.nseg) * (SUMMARY_STRIDE / 4) : nullptr, g, hi, v, a, s_addr, sb_addr,
                                 0, init_shared ? 2 : 4);
                 tc_wait_st();
@@ -510,7 +510,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         outputs(nc - 1);
         mbar_wait(&sh.u_full[hi], (nc - 1) & 1, abortp, p.status);
         tc_fence_after();
-        if (g == sq.last_seg) store_state(slot1 + (size_t)hi * state_stride, v, s_addr, 0, 4);
+        if (g == sq.last_seg && !(p.single && hi == 1)) store_state(slot1 + (size_t)hi * state_stride, v, s_addr, 0, 4);
     }
     tc_fence_before();
     __syncthreads();

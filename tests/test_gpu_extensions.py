@@ -175,8 +175,8 @@ def test_tensor_kernels_refuse_per_key_channel_gates():
 @pytest.mark.parametrize("dtype,d,vec,impl", [(F32, 64, False, "auto"), (BF, 128, False, "auto"), (BF, 128, False, "simt"), (BF, 128, True, "auto"),
                                                (F32, 64, True, "auto")])
 def test_nstate_prefill(n, dtype, d, vec, impl):
-    """bf16, d = 128, scalar gates, even n: AUTO runs the chunkwise tensor-core kernel once per pair of states; everything
-    else (and impl="simt") the token-by-token kernel."""
+    """bf16, d = 128, scalar gates: AUTO runs the chunkwise tensor-core kernel once per pair of states (n = 1: a pair whose
+    second state has weight 0 and never touches the slot); everything else (and impl="simt") the token-by-token kernel."""
     import paper_2506_09316_b200 as dsla
     rng = np.random.default_rng(3700 + n + d)
     lens = [33, 0, 150, 1]
@@ -204,7 +204,7 @@ def test_nstate_prefill(n, dtype, d, vec, impl):
     assert rel_err(_f64(st.tensor), S_ref) <= TOL[dtype]
 
 
-@pytest.mark.parametrize("n,use_init", [(2, False), (4, True), (8, False)])
+@pytest.mark.parametrize("n,use_init", [(1, True), (1, False), (2, False), (4, True), (8, False)])
 def test_nstate_prefill_tensor_path_with_split_sequences(n, use_init):
     """Few (sequence, head) pairs and long sequences: every pair of states runs the summary pass, the fold and (on a
     resume) the snapshot of its own two states; pairs after the first add to the output."""
@@ -232,9 +232,9 @@ def test_nstate_prefill_tensor_path_with_split_sequences(n, use_init):
     assert rel_err(_f64(o), o_ref) <= TOL[BF] * (1.5 if n == 8 else 1.0)
     assert rel_err(_f64(st.tensor), S_ref) <= TOL[BF]
     # the tensor path is refused where it does not apply
-    with pytest.raises(dsla.DslaError) as e:
-        dsla.dsla_nstate_prefill(dv.q, dv.k, dv.v, torch.ones(1, T, H, device="cuda"), torch.ones(H, 1, device="cuda"),
-                                 dsla.dsla_state_alloc_n(3, 1, H, d, d), cu_seqlens=dv.cu_seqlens, max_seqlen=max(lens), impl="tensor")
+    with pytest.raises(dsla.DslaError) as e:        # gates per key channel
+        dsla.dsla_nstate_prefill(dv.q, dv.k, dv.v, torch.ones(n, T, H, d, device="cuda"), torch.from_numpy(w).cuda(), st,
+                                 cu_seqlens=dv.cu_seqlens, max_seqlen=max(lens), impl="tensor")
     assert e.value.status == dsla.DSLA_ERR_UNSUPPORTED
 
 
